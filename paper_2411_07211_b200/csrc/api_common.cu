@@ -1,0 +1,67 @@
+// Library-wide pieces: workspace helpers, status strings, tuning knobs, device queries.
+#include "common.cuh"
+
+namespace b2 {
+
+static int64_t g_knobs[kKnobCount] = {
+    /* kKnobL1BlocksPerSm   */ 8,
+    /* kKnobGemvNTileBytes  */ 64 * 1024,
+    /* kKnobGemvTRows       */ 256,
+    /* kKnobTriRows         */ 256,
+    /* kKnobGerRows         */ 2,
+    /* kKnobUsePdl          */ 1,
+    /* kKnobTrsvDebugSkip   */ -1,
+    /* kKnobTriWide         */ 0,
+};
+
+int64_t knob(int id) { return (id >= 0 && id < kKnobCount) ? g_knobs[id] : 0; }
+
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+}  // namespace b2
+
+extern "C" {
+
+size_t b2_workspace_min_bytes(void) { return b2::kCtlBytes + 64 * 1024; }
+size_t b2_workspace_bytes(void) { return (size_t)64 << 20; }
+
+int b2_workspace_reset(const b2_ctx* ctx) {
+  b2::Launch l;
+  if (int st = b2::make_launch(ctx, &l)) return st;
+  return cudaMemsetAsync(ctx->workspace, 0, b2::kCtlBytes, l.stream) == cudaSuccess ? B2_STATUS_OK
+                                                                                    : B2_STATUS_LAUNCH_FAILED;
+}
+
+const char* b2_status_string(int status) {
+  if (status < 0) return "invalid argument (the negated value is its 1-based position after ctx)";
+  switch (status) {
+    case B2_STATUS_OK: return "ok";
+    case B2_STATUS_LAUNCH_FAILED: return "CUDA launch failed";
+    case B2_STATUS_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case B2_STATUS_NOT_IMPLEMENTED: return "not implemented";
+    case B2_STATUS_TIMEOUT: return "a bounded device-side wait ran out";
+    case B2_STATUS_BAD_CONTEXT: return "bad context (NULL, or workspace NULL / not 256-byte aligned)";
+    default: return "unknown status";
+  }
+}
+
+int b2_version(void) { return 100; }
+
+int b2_set_tuning(int knob_id, int64_t value) {
+  if (knob_id < 0 || knob_id >= b2::kKnobCount) return -1;
+  b2::g_knobs[knob_id] = value;
+  return 0;
+}
+int64_t b2_get_tuning(int knob_id) { return b2::knob(knob_id); }
+
+}  // extern "C"

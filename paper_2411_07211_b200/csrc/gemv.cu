@@ -1,0 +1,62 @@
+// gemv entry points: y <- alpha*op(A)*x + beta*y (Section 2 inset and Figure 7 of the paper).
+// Row-major N is the row-dot kind, row-major T the column-sum kind; a column-major call is
+// the transposed row-major problem (A^T stored row-major), so N and T swap kinds.
+#include "level2.cuh"
+
+namespace b2 {
+
+using GemvRow = Kind<true, false, TRI_FULL, false, false>;
+using GemvCol = Kind<false, true, TRI_FULL, false, false>;
+
+template <typename T>
+static int gemv_impl(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t n, T alpha, const T* a, int64_t lda,
+                     const T* x, int64_t incx, T beta, T* y, int64_t incy) {
+  if (order != B2_ROW_MAJOR && order != B2_COL_MAJOR) return -1;
+  if (trans != B2_NO_TRANS && trans != B2_TRANS) return -2;
+  if (m < 0) return -3;
+  if (n < 0) return -4;
+  const int64_t minor = order == B2_ROW_MAJOR ? n : m;
+  if (m > 0 && n > 0 && (a == nullptr || !aligned_to(a, sizeof(T)))) return -6;
+  if (lda < (minor > 1 ? minor : 1)) return -7;
+  const int64_t lenx = trans == B2_NO_TRANS ? n : m, leny = trans == B2_NO_TRANS ? m : n;
+  if (incx == 0) return -9;
+  if (lenx > 0 && leny > 0 && (x == nullptr || !aligned_to(x, sizeof(T)))) return -8;
+  if (incy == 0) return -12;
+  if (leny > 0 && (y == nullptr || !aligned_to(y, sizeof(T)))) return -11;
+  Launch l;
+  if (int st = make_launch(ctx, &l)) return st;
+  if (m == 0 || n == 0) return B2_STATUS_OK;
+  if (alpha == T(0)) return scale_y<T>(l, y, incy, leny, beta);
+
+  L2Args<T> args = {};
+  args.a = a;
+  args.lda = lda;
+  args.rows = order == B2_ROW_MAJOR ? m : n;  // canonical row-major view
+  args.cols = order == B2_ROW_MAJOR ? n : m;
+  args.alpha = alpha;
+  args.beta = beta;
+  args.y = vec_base(y, leny, incy);
+  args.incy = incy;
+  const bool rowdot = (order == B2_ROW_MAJOR) == (trans == B2_NO_TRANS);
+  if (rowdot) {
+    args.xc = vec_base(x, lenx, incx);
+    args.incxc = incx;
+    return l2_dispatch<T, GemvRow, true>(l, args, plan_rowout(args, true), true);
+  }
+  args.xr = vec_base(x, lenx, incx);
+  args.incxr = incx;
+  return l2_dispatch<T, GemvCol, true>(l, args, plan_colout(args, true, knob(kKnobGemvTRows)), true);
+}
+
+}  // namespace b2
+
+extern "C" {
+int b2_sgemv(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t n, float alpha, const float* a, int64_t lda,
+             const float* x, int64_t incx, float beta, float* y, int64_t incy) {
+  return b2::gemv_impl<float>(ctx, order, trans, m, n, alpha, a, lda, x, incx, beta, y, incy);
+}
+int b2_dgemv(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t n, double alpha, const double* a, int64_t lda,
+             const double* x, int64_t incx, double beta, double* y, int64_t incy) {
+  return b2::gemv_impl<double>(ctx, order, trans, m, n, alpha, a, lda, x, incx, beta, y, incy);
+}
+}

@@ -1,0 +1,100 @@
+// symv and trmv entry-point bodies (Section 6.2.2, "Triangular Matrix"): both run on the
+// level-2 tile kernel restricted to one triangle of the canonical row-major view.
+//   symv : row sums over the stored triangle (with the diagonal) plus column sums over its
+//          strictly off-diagonal part -- each stored element is loaded once and used twice.
+//   trmv : row sums (op(A) rows contiguous) or column sums (op(A) rows strided), the
+//          diagonal replaced by 1 for diag = unit.  The result goes to partials first and is
+//          written over x by the finalize kernel, after every block has finished reading x.
+#pragma once
+#include "level2.cuh"
+
+namespace b2 {
+
+template <typename T>
+static int check_square(int order, int64_t n, const T* a, int64_t lda, int arg_order, int arg_n, int arg_a,
+                        int arg_lda) {
+  if (order != B2_ROW_MAJOR && order != B2_COL_MAJOR) return -arg_order;
+  if (n < 0) return -arg_n;
+  if (n > 0 && (a == nullptr || !aligned_to(a, sizeof(T)))) return -arg_a;
+  if (lda < (n > 1 ? n : 1)) return -arg_lda;
+  return 0;
+}
+
+template <typename T>
+static L2Plan plan_tri(const L2Args<T>& a) {
+  const int V = (aligned_to(a.a, 16) && a.lda % VecLen<T>::value == 0) ? VecLen<T>::value : 1;
+  const int64_t nv = (a.cols + V - 1) / V;
+  L2Plan p;
+  p.shape = (nv >= 512 && knob(kKnobTriWide)) ? SHAPE_WIDE : SHAPE_MID;
+  p.ctiles_per_cta = 1;
+  p.rows_per_cta = knob(kKnobTriRows);
+  return p;
+}
+
+template <typename T>
+static int symv_impl(const b2_ctx* ctx, int order, int uplo, int64_t n, T alpha, const T* a, int64_t lda, const T* x,
+                     int64_t incx, T beta, T* y, int64_t incy) {
+  if (int e = check_square(order, n, a, lda, 1, 3, 5, 6)) return e;
+  if (uplo != B2_UPPER && uplo != B2_LOWER) return -2;
+  if (incx == 0) return -8;
+  if (n > 0 && (x == nullptr || !aligned_to(x, sizeof(T)))) return -7;
+  if (incy == 0) return -11;
+  if (n > 0 && (y == nullptr || !aligned_to(y, sizeof(T)))) return -10;
+  Launch l;
+  if (int st = make_launch(ctx, &l)) return st;
+  if (n == 0) return B2_STATUS_OK;
+  if (alpha == T(0)) return scale_y<T>(l, y, incy, n, beta);
+  L2Args<T> args = {};
+  args.a = a;
+  args.lda = lda;
+  args.rows = args.cols = n;
+  args.xc = args.xr = vec_base(x, n, incx);
+  args.incxc = args.incxr = incx;
+  args.alpha = alpha;
+  args.beta = beta;
+  args.y = vec_base(y, n, incy);
+  args.incy = incy;
+  // the stored triangle as it sits in the row-major view of the buffer
+  const bool upper = (order == B2_ROW_MAJOR) == (uplo == B2_UPPER);
+  const L2Plan plan = plan_tri(args);
+  if (upper) return l2_dispatch<T, Kind<true, true, TRI_UPPER, false, true>, false>(l, args, plan, false);
+  return l2_dispatch<T, Kind<true, true, TRI_LOWER, false, true>, false>(l, args, plan, false);
+}
+
+template <typename T, bool ROW, int TRI>
+static int trmv_kind(const Launch& l, const L2Args<T>& args, bool unit) {
+  const L2Plan plan = ROW ? plan_rowout(args, false) : plan_colout(args, false, knob(kKnobTriRows));
+  if (unit) return l2_dispatch<T, Kind<ROW, !ROW, TRI, true, false>, false>(l, args, plan, false);
+  return l2_dispatch<T, Kind<ROW, !ROW, TRI, false, false>, false>(l, args, plan, false);
+}
+
+template <typename T>
+static int trmv_impl(const b2_ctx* ctx, int order, int uplo, int trans, int diag, int64_t n, const T* a, int64_t lda,
+                     T* x, int64_t incx) {
+  if (int e = check_square(order, n, a, lda, 1, 5, 6, 7)) return e;
+  if (uplo != B2_UPPER && uplo != B2_LOWER) return -2;
+  if (trans != B2_NO_TRANS && trans != B2_TRANS) return -3;
+  if (diag != B2_NON_UNIT && diag != B2_UNIT) return -4;
+  if (incx == 0) return -9;
+  if (n > 0 && (x == nullptr || !aligned_to(x, sizeof(T)))) return -8;
+  Launch l;
+  if (int st = make_launch(ctx, &l)) return st;
+  if (n == 0) return B2_STATUS_OK;
+  L2Args<T> args = {};
+  args.a = a;
+  args.lda = lda;
+  args.rows = args.cols = n;
+  args.xc = args.xr = vec_base(x, n, incx);
+  args.incxc = args.incxr = incx;
+  args.alpha = T(1);
+  args.beta = T(0);
+  args.y = vec_base(x, n, incx);
+  args.incy = incx;
+  const bool upper = (order == B2_ROW_MAJOR) == (uplo == B2_UPPER);
+  const bool row = (order == B2_ROW_MAJOR) == (trans == B2_NO_TRANS);
+  const bool unit = diag == B2_UNIT;
+  if (row) return upper ? trmv_kind<T, true, TRI_UPPER>(l, args, unit) : trmv_kind<T, true, TRI_LOWER>(l, args, unit);
+  return upper ? trmv_kind<T, false, TRI_UPPER>(l, args, unit) : trmv_kind<T, false, TRI_LOWER>(l, args, unit);
+}
+
+}  // namespace b2
