@@ -77,6 +77,8 @@ size_t b2_workspace_bytes(void);     /* recommended size (64 MiB)               
 int b2_workspace_reset(const b2_ctx* ctx); /* async memset of the control block to zero     */
 const char* b2_status_string(int status);
 int b2_version(void);
+/* Number of kernels this library has launched in this process so far (not thread-safe). */
+unsigned long long b2_launch_count(void);
 
 /* Tuning hooks (process-wide, not thread-safe): work-splitting parameters of the kernels,
  * indexed by the Knob enumeration of the sources.  Defaults are the tuned values; changing

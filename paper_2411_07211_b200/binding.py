@@ -87,6 +87,7 @@ def lib():
         h.b2_status_string.restype = ctypes.c_char_p
         h.b2_status_string.argtypes = [_int]
         h.b2_version.restype = _int
+        h.b2_launch_count.restype = ctypes.c_ulonglong
         h.b2_set_tuning.argtypes = [_int, _i64]
         h.b2_set_tuning.restype = _int
         h.b2_get_tuning.argtypes = [_int]
@@ -97,7 +98,7 @@ def lib():
 
 def exported_symbols():
     return sorted(_protos().keys()) + ["b2_workspace_min_bytes", "b2_workspace_bytes", "b2_status_string",
-                                       "b2_version", "b2_set_tuning", "b2_get_tuning"]
+                                       "b2_version", "b2_launch_count", "b2_set_tuning", "b2_get_tuning"]
 
 
 class Context:
@@ -222,3 +223,7 @@ def set_tuning(knob: int, value: int):
 
 def get_tuning(knob: int) -> int:
     return int(lib().b2_get_tuning(knob))
+
+
+def launch_count() -> int:
+    return int(lib().b2_launch_count())

@@ -14,6 +14,8 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobTriWide         */ 0,
 };
 
+unsigned long long g_launch_count = 0;
+
 int64_t knob(int id) { return (id >= 0 && id < kKnobCount) ? g_knobs[id] : 0; }
 
 int sm_count() {
@@ -56,6 +58,8 @@ const char* b2_status_string(int status) {
 }
 
 int b2_version(void) { return 100; }
+
+unsigned long long b2_launch_count(void) { return b2::g_launch_count; }
 
 int b2_set_tuning(int knob_id, int64_t value) {
   if (knob_id < 0 || knob_id >= b2::kKnobCount) return -1;

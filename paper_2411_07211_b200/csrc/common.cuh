@@ -133,7 +133,12 @@ inline int make_launch(const b2_ctx* ctx, Launch* l) {
   return B2_STATUS_OK;
 }
 
-inline int check_launch() { return cudaGetLastError() == cudaSuccess ? B2_STATUS_OK : B2_STATUS_LAUNCH_FAILED; }
+// Every kernel launch site calls this right after the launch; it also feeds the launch counter.
+extern unsigned long long g_launch_count;
+inline int check_launch() {
+  ++g_launch_count;
+  return cudaGetLastError() == cudaSuccess ? B2_STATUS_OK : B2_STATUS_LAUNCH_FAILED;
+}
 
 // Number of SMs of the current device (cached per device id).
 int sm_count();
