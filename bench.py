@@ -1,0 +1,510 @@
+#!/usr/bin/env python
+"""Benchmark of the BLAS level-1/2 family: achieved HBM GB/s per variant and their geomean.
+
+A "step" is one pass over the whole variant cross-product (every routine x {f32, f64} x
+trans/uplo/diag options x inc in {1, 2}), each variant sized to a 256 MiB working set.  Every
+variant is timed with its own pair of CUDA events on the launching stream; L2 is flushed
+(256 MiB memset) before each variant so no number is an L2-resident one.  Prints ONE JSON
+line (rank 0).
+
+    python bench.py --gpus 1 --steps 20 --warmup 3
+    python bench.py --impl reference        # the CPU oracle on the host cores (bounded sample)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+MIB = 1 << 20
+ROW, COL, NOTR, TR, UP, LO, NONU, UNIT = 101, 102, 111, 112, 121, 122, 131, 132
+FALLBACK_PEAK_GBS = 6650.0
+
+
+# --------------------------------------------------------------------------- variant table
+def variant_specs(scale: int = 1):
+    """The cross-product.  `scale` divides the element counts (used by the CPU legs).
+    Each spec: name, family (kernel template), routine, dtype, options, sizes, bytes."""
+    specs = []
+    for dt, s in (("f32", 4), ("f64", 8)):
+        for inc in (1, 2):
+            n2 = (128 * MIB // s) // inc // scale  # two-vector routines: 2 x 128 MiB spans
+            n1 = (256 * MIB // s) // inc // scale  # one-vector routines: one 256 MiB span
+            for r, per_elem, nvec in (("axpy", 3, 2), ("scal", 2, 1), ("copy", 2, 2), ("swap", 4, 2), ("rot", 4, 2),
+                                      ("dot", 2, 2), ("asum", 1, 1), ("nrm2", 1, 1), ("iamax", 1, 1)):
+                n = n2 if nvec == 2 else n1
+                fam = "l1_map" if r in ("axpy", "scal", "copy", "swap", "rot") else "l1_reduce"
+                specs.append(dict(name=f"{r}_{dt}_inc{inc}", family=fam, routine=r, dtype=dt, inc=inc, n=n,
+                                  useful=per_elem * n * s, touched=per_elem * n * s * inc))
+        ng = (8192 if s == 4 else 5760) // int(math.isqrt(scale))
+        nt = (11520 if s == 4 else 8192) // int(math.isqrt(scale))
+        for inc in (1, 2):
+            vec = ng * s * inc
+            for tr, tn in ((NOTR, "n"), (TR, "t")):
+                specs.append(dict(name=f"gemv_{tn}_{dt}_inc{inc}", family="l2_tile", routine="gemv", dtype=dt, inc=inc,
+                                  n=ng, trans=tr, useful=(ng * ng + 3 * ng) * s, touched=ng * ng * s + 3 * vec))
+            specs.append(dict(name=f"ger_{dt}_inc{inc}", family="ger", routine="ger", dtype=dt, inc=inc, n=ng,
+                              useful=(2 * ng * ng + 2 * ng) * s, touched=2 * ng * ng * s + 2 * vec))
+            tri = nt * (nt + 1) // 2
+            tvec = nt * s * inc
+            for ul, un in ((UP, "u"), (LO, "l")):
+                specs.append(dict(name=f"symv_{un}_{dt}_inc{inc}", family="l2_tile", routine="symv", dtype=dt, inc=inc,
+                                  n=nt, uplo=ul, useful=(tri + 3 * nt) * s, touched=tri * s + 3 * tvec))
+                for tr, tn in ((NOTR, "n"), (TR, "t")):
+                    for dg, dn in ((NONU, "n"), (UNIT, "u")):
+                        t = tri - (nt if dg == UNIT else 0)
+                        for r, fam in (("trmv", "l2_tile"), ("trsv", "trsv")):
+                            specs.append(dict(name=f"{r}_{un}{tn}{dn}_{dt}_inc{inc}", family=fam, routine=r, dtype=dt,
+                                              inc=inc, n=nt, uplo=ul, trans=tr, diag=dg,
+                                              useful=(t + 2 * nt) * s, touched=t * s + 2 * tvec))
+    return specs
+
+
+def geomean(vals):
+    vals = [v for v in vals if v > 0]
+    return math.exp(sum(math.log(v) for v in vals) / len(vals)) if vals else 0.0
+
+
+def peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_PEAK_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+# --------------------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        self.lines = []
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- GPU arm
+class GpuWorkload:
+    """Device buffers (seeded synthetic data) and one launcher per variant."""
+
+    def __init__(self, device):
+        import torch
+        from paper_2411_07211_b200 import binding as b2
+        from paper_2411_07211_b200 import synth
+        self.torch, self.b2, self.synth = torch, b2, synth
+        self.dev = device
+        self.ctx = b2.Context(device)
+        self.ctx.reset()
+        self.specs = variant_specs()
+        self.flush = torch.empty(256 * MIB, dtype=torch.uint8, device=device)
+        tdt = {"f32": torch.float32, "f64": torch.float64}
+        self.buf = {}
+        for dt, s in (("f32", 4), ("f64", 8)):
+            t = tdt[dt]
+            nel = 256 * MIB // s
+            # level-1 vectors: X is a 256 MiB span, Y a 128 MiB span (+1 so inc=2 spans fit)
+            self.buf[dt, "x"] = synth.vector_torch(0, 10, nel, t, device)
+            self.buf[dt, "y"] = synth.vector_torch(0, 11, nel // 2, t, device)
+            ng = 8192 if s == 4 else 5760
+            nt = 11520 if s == 4 else 8192
+            self.buf[dt, "ag"] = synth.matrix_torch(0, 12, ng, ng, ng, t, device)
+            self.buf[dt, "ager"] = synth.matrix_torch(0, 13, ng, ng, ng, t, device)
+            self.buf[dt, "at"] = synth.matrix_torch(0, 14, nt, nt, nt, t, device, tri_n=nt)
+            nv = max(ng, nt)
+            self.buf[dt, "vx0"] = synth.vector_torch(0, 15, 2 * nv, t, device)  # pristine copies
+            self.buf[dt, "vy0"] = synth.vector_torch(0, 16, 2 * nv, t, device)
+            self.buf[dt, "vx"] = self.buf[dt, "vx0"].clone()
+            self.buf[dt, "vy"] = self.buf[dt, "vy0"].clone()
+            self.buf[dt, "res"] = torch.zeros(4, dtype=t, device=device)
+        self.ires = torch.zeros(1, dtype=torch.int64, device=device)
+        torch.cuda.synchronize(device)
+
+    def restore(self, sp):
+        """Puts back vectors that a previous in-place call changed (tiny; uses the library's own
+        copy kernel, outside the variant's event bracket)."""
+        if sp["routine"] in ("trmv", "trsv"):
+            B, dt = self.buf, sp["dtype"]
+            self.b2.copy(self.ctx, 2 * sp["n"], B[dt, "vx0"], 1, B[dt, "vx"], 1)
+
+    def launch(self, sp):
+        b2, ctx, B = self.b2, self.ctx, self.buf
+        dt, inc, n, r = sp["dtype"], sp["inc"], sp["n"], sp["routine"]
+        x, y, res = B[dt, "x"], B[dt, "y"], B[dt, "res"]
+        if r == "axpy":
+            b2.axpy(ctx, n, 1.5, x, inc, y, inc)
+        elif r == "scal":
+            b2.scal(ctx, n, -0.75, x, inc)
+        elif r == "copy":
+            b2.copy(ctx, n, x, inc, y, inc)
+        elif r == "swap":
+            b2.swap(ctx, n, x, inc, y, inc)
+        elif r == "rot":
+            b2.rot(ctx, n, x, inc, y, inc, 0.6, 0.8)
+        elif r == "dot":
+            b2.dot(ctx, n, x, inc, y, inc, res[0:1])
+        elif r == "asum":
+            b2.asum(ctx, n, x, inc, res[1:2])
+        elif r == "nrm2":
+            b2.nrm2(ctx, n, x, inc, res[2:3])
+        elif r == "iamax":
+            b2.iamax(ctx, n, x, inc, self.ires)
+        elif r == "gemv":
+            b2.gemv(ctx, ROW, sp["trans"], n, n, 1.25, B[dt, "ag"], n, B[dt, "vx"], inc, 0.5, B[dt, "vy"], inc)
+        elif r == "ger":
+            b2.ger(ctx, ROW, n, n, 1.25, B[dt, "vx0"], inc, B[dt, "vy0"], inc, B[dt, "ager"], n)
+        elif r == "symv":
+            b2.symv(ctx, ROW, sp["uplo"], n, 1.25, B[dt, "at"], n, B[dt, "vx0"], inc, 0.5, B[dt, "vy"], inc)
+        elif r == "trmv":
+            b2.trmv(ctx, ROW, sp["uplo"], sp["trans"], sp["diag"], n, B[dt, "at"], n, B[dt, "vx"], inc)
+        elif r == "trsv":
+            b2.trsv(ctx, ROW, sp["uplo"], sp["trans"], sp["diag"], n, B[dt, "at"], n, B[dt, "vx"], inc)
+        else:
+            raise KeyError(r)
+
+    def step(self, events=None):
+        """One pass over every variant; `events` (list of (start, end) pairs) brackets each."""
+        for k, sp in enumerate(self.specs):
+            self.flush.zero_()  # L2 flush: 256 MiB write
+            self.restore(sp)
+            if events is not None:
+                events[k][0].record()
+            self.launch(sp)
+            if events is not None:
+                events[k][1].record()
+
+
+def e2e_leg(wl: GpuWorkload, steps: int):
+    """Same metric through the C ABI with HOST data: per variant, pinned host -> device copies of
+    its inputs, the call, and a device -> host read of its outputs, all inside the timed bracket."""
+    torch, B = wl.torch, wl.buf
+    pinned = {}
+
+    def pin(key):
+        """One pinned host mirror per device buffer (inputs are read from it, outputs land in it)."""
+        if key not in pinned:
+            t = dev(key)
+            pinned[key] = torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+        return pinned[key]
+
+    def io(sp):
+        dt, r = sp["dtype"], sp["routine"]
+        v = ("x", "y") if sp["family"] in ("l1_map", "l1_reduce") else ("vx", "vy")
+        ins, outs = [], []
+        if r in ("axpy", "swap", "rot", "dot"):
+            ins = [v[0], v[1]]
+        elif r in ("scal", "copy", "asum", "nrm2", "iamax"):
+            ins = [v[0]]
+        elif r == "gemv":
+            ins = ["ag", "vx", "vy"]
+        elif r == "ger":
+            ins = ["ager", "vx0", "vy0"]
+        elif r == "symv":
+            ins = ["at", "vx0", "vy"]
+        else:
+            ins = ["at", "vx"]
+        outs = {"axpy": ["y"], "scal": ["x"], "copy": ["y"], "swap": ["x", "y"], "rot": ["x", "y"], "dot": ["res"],
+                "asum": ["res"], "nrm2": ["res"], "iamax": ["ires"], "gemv": ["vy"], "ger": ["ager"],
+                "symv": ["vy"], "trmv": ["vx"], "trsv": ["vx"]}[r]
+        return [(dt, k) for k in ins], [(dt, k) for k in outs]
+
+    def sl(sp, key, t):
+        """The part of a buffer this variant really uses (so copies are not oversized)."""
+        if key[1] in ("x", "y"):
+            return t[: (sp["n"] - 1) * sp["inc"] + 1]
+        if key[1] in ("vx", "vy", "vx0", "vy0"):
+            return t[: (sp["n"] - 1) * sp["inc"] + 1]
+        return t
+
+    def dev(key):
+        return wl.ires if key[1] == "ires" else B[key]
+
+    per_variant = [[] for _ in wl.specs]
+    h2d = d2h = 0
+    for it in range(steps + 1):  # first pass is warm-up (also pins the host copies)
+        h2d = d2h = 0
+        for k, sp in enumerate(wl.specs):
+            ins, outs = io(sp)
+            hin = [(key, sl(sp, key, pin(key))) for key in ins]
+            hout = [(key, sl(sp, key, pin(key))) for key in outs]
+            wl.flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for key, h in hin:
+                sl(sp, key, dev(key)).copy_(h, non_blocking=True)
+                h2d += h.numel() * h.element_size()
+            wl.launch(sp)
+            for key, h in hout:
+                h.copy_(sl(sp, key, dev(key)), non_blocking=True)
+                d2h += h.numel() * h.element_size()
+            e1.record()
+            e1.synchronize()
+            if it > 0:
+                per_variant[k].append(e0.elapsed_time(e1))
+    med = [sorted(v)[len(v) // 2] for v in per_variant]
+    gbs = [sp["touched"] / (t * 1e-3) / 1e9 for sp, t in zip(wl.specs, med)]
+    return {"value": geomean(gbs), "unit": "GB/s (geomean over variants, host buffers in and out)",
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps}
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+def oracle_pass(scale: int, seed: int = 0):
+    """Times the CPU oracle, as it stands, over every variant at 1/scale of the bench's element
+    counts.  Returns per-variant GB/s (touched bytes of the SAMPLE / oracle seconds)."""
+    import numpy as np
+    from oracle import blas_oracle as orc
+    from paper_2411_07211_b200 import synth
+    out = []
+    cache = {}
+
+    def vec(dt, stream, n):
+        key = (dt, stream, n)
+        if key not in cache:
+            cache[key] = synth.vector_np(seed, stream, n, np.float32 if dt == "f32" else np.float64)
+        return cache[key]
+
+    for sp in variant_specs(scale):
+        dt, inc, n, r = sp["dtype"], sp["inc"], sp["n"], sp["routine"]
+        npdt = np.float32 if dt == "f32" else np.float64
+        if sp["family"] in ("l1_map", "l1_reduce"):
+            x = vec(dt, 10, (n - 1) * inc + 1).copy()
+            y = vec(dt, 11, (n - 1) * inc + 1).copy()
+            fn = {"axpy": lambda: orc.axpy(n, npdt(1.5), x, inc, y, inc), "scal": lambda: orc.scal(n, npdt(-0.75), x, inc),
+                  "copy": lambda: orc.copy(n, x, inc, y, inc), "swap": lambda: orc.swap(n, x, inc, y, inc),
+                  "rot": lambda: orc.rot(n, x, inc, y, inc, npdt(0.6), npdt(0.8)),
+                  "dot": lambda: orc.dot(n, x, inc, y, inc), "asum": lambda: orc.asum(n, x, inc),
+                  "nrm2": lambda: orc.nrm2(n, x, inc), "iamax": lambda: orc.iamax(n, x, inc)}[r]
+        else:
+            key = (dt, "mat", n, r in ("symv", "trmv", "trsv"))
+            if key not in cache:
+                cache[key] = synth.matrix_np(seed, 14, n, n, n, npdt, tri_n=n if key[3] else None).ravel()
+            a = cache[key]
+            x = vec(dt, 15, (n - 1) * inc + 1).copy()
+            y = vec(dt, 16, (n - 1) * inc + 1).copy()
+            if r == "gemv":
+                fn = lambda: orc.gemv(ROW, sp["trans"], n, n, npdt(1.25), a, n, x, inc, npdt(0.5), y, inc)
+            elif r == "ger":
+                a = a.copy()
+                fn = lambda: orc.ger(ROW, n, n, npdt(1.25), x, inc, y, inc, a, n, want_absterms=False)
+            elif r == "symv":
+                fn = lambda: orc.symv(ROW, sp["uplo"], n, npdt(1.25), a, n, x, inc, npdt(0.5), y, inc)
+            elif r == "trmv":
+                fn = lambda: orc.trmv(ROW, sp["uplo"], sp["trans"], sp["diag"], n, a, n, x, inc)
+            else:
+                fn = lambda: orc.trsv(ROW, sp["uplo"], sp["trans"], sp["diag"], n, a, n, x, inc)
+        t0 = time.perf_counter()
+        fn()
+        dt_s = time.perf_counter() - t0
+        out.append((sp["name"], sp["touched"] / dt_s / 1e9, dt_s))
+    return out
+
+
+def reference_arm(args):
+    """`--impl reference`: the oracle, as it stands, on the host cores; each step is one pass over
+    every variant at 1/64 of the bench's element counts (bounded so the run ends in minutes)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    scale = 16
+    from oracle import blas_oracle as orc
+    orc.build()
+    for _ in range(args.warmup):
+        oracle_pass(scale)
+    t0 = time.perf_counter()
+    runs = [oracle_pass(scale) for _ in range(args.steps)]
+    wall = time.perf_counter() - t0
+    per = [geomean([run[k][1] for run in runs]) for k in range(len(runs[0]))]
+    value = geomean(per)
+    sample = f"every variant at 1/{scale} of the bench element counts (16 MiB working sets), 1 thread"
+    print(json.dumps({
+        "impl": "reference", "metric": "achieved GB/s per BLAS-1/2 variant, geomean over variants",
+        "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": wall / max(1, args.steps) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32+f64", "data": "synthetic",
+        "config": {"workload": "config 5 cross-product (routines x f32/f64 x options x inc 1/2), CPU sample",
+                   "variants": len(per)},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# --------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--table", default=None, help="also write the per-variant table (JSON) to this path")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2411_07211_b200 import binding as b2
+    wl = GpuWorkload(device)
+    nv = len(wl.specs)
+    warm = max(3, args.warmup)
+    for _ in range(warm):
+        wl.step()
+    torch.cuda.synchronize(device)
+    events = [[[torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)] for _ in range(nv)]
+              for _ in range(args.steps)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize(device)
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = b2.launch_count()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for s in range(args.steps):
+        wl.step(events[s])
+    t_end.record()
+    torch.cuda.synchronize(device)
+    if world > 1:
+        dist.barrier()
+    launches = b2.launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    total_ms = t_start.elapsed_time(t_end)
+    assert wl.ctx.device_status() == 0, "a trsv wait timed out during the bench"
+
+    med = []
+    for k in range(nv):
+        ts = sorted(events[s][k][0].elapsed_time(events[s][k][1]) for s in range(args.steps))
+        med.append(ts[len(ts) // 2])
+    times = torch.tensor(med + [total_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    times = times.cpu().tolist()
+    med, total_ms = times[:-1], times[-1]
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = peak_gbs()
+    rows = []
+    for sp, t in zip(wl.specs, med):
+        gbs = world * sp["touched"] / (t * 1e-3) / 1e9
+        rows.append({"name": sp["name"], "family": sp["family"], "ms": t, "gbs": gbs / world,
+                     "gbs_useful": sp["useful"] / (t * 1e-3) / 1e9, "frac": gbs / world / peak})
+    value = world * geomean([r["gbs"] for r in rows])
+    fam = {}
+    for sp, r in zip(wl.specs, rows):
+        f = fam.setdefault(sp["family"], {"ms": 0.0, "bytes": 0, "launches": 0})
+        f["ms"] += r["ms"]
+        f["bytes"] += sp["touched"]
+        f["launches"] += 1
+    by_kernel = {k: {"achieved": v["bytes"] / (v["ms"] * 1e-3) / 1e9, "frac": v["bytes"] / (v["ms"] * 1e-3) / 1e9 / peak,
+                     "share_of_time": v["ms"] / sum(x["ms"] for x in fam.values()), "variants": v["launches"]}
+                 for k, v in fam.items()}
+    dom = max(fam, key=lambda k: fam[k]["ms"])
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    traffic = None
+    try:
+        traffic = json.load(open(traffic_path)).get(dom)
+    except Exception:
+        pass
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": by_kernel[dom]["achieved"], "peak": peak, "unit": "GB/s",
+                "frac": by_kernel[dom]["frac"], "traffic": traffic, "peak_source": peak_src,
+                "by_kernel": by_kernel}
+    no_trsv = [r for r in rows if r["family"] != "trsv"]
+    out = {
+        "metric": "achieved HBM GB/s per BLAS-1/2 variant, geomean over variants",
+        "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32+f64", "data": "synthetic",
+        "config": {"workload": "config 5: every routine x {f32,f64} x trans/uplo/diag x inc {1,2}, 256 MiB working "
+                               "set per variant, row-major", "variants": nv,
+                   "l2": "flushed before every variant (256 MiB memset)", "bytes": "touched sectors (span bytes)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "geomean_frac_of_peak": value / world / peak,
+        "geomean_frac_of_peak_without_trsv": geomean([r["frac"] for r in no_trsv]),
+        "geomean_frac_by_family": {k: geomean([r["frac"] for r in rows if r["family"] == k]) for k in fam},
+        "min_variant": min(rows, key=lambda r: r["frac"])["name"],
+        "gpu_launches": launches, "clocks": clocks, "roofline": roofline,
+    }
+    if not args.no_e2e and world == 1:
+        out["e2e"] = e2e_leg(wl, min(args.steps, 2))
+    else:
+        out["e2e"] = None
+    if not args.no_cpu and world == 1:
+        scale = 16
+        t0 = time.perf_counter()
+        res = oracle_pass(scale)
+        out["cpu_baseline"] = {"value": geomean([r[1] for r in res]), "unit": "GB/s", "cores": 1, "kind": "oracle",
+                               "sample": f"every variant once at 1/{scale} of the bench element counts "
+                                         f"({time.perf_counter() - t0:.1f} s of CPU work)"}
+    else:
+        out["cpu_baseline"] = None
+    out["variants"] = [{k: (round(v, 4) if isinstance(v, float) else v) for k, v in r.items()} for r in rows]
+    if args.table:
+        os.makedirs(os.path.dirname(os.path.abspath(args.table)), exist_ok=True)
+        with open(args.table, "w") as f:
+            json.dump(out, f, indent=1)
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
