@@ -47,7 +47,8 @@ enum {
   B2_STATUS_WORKSPACE_TOO_SMALL = 2, /* ctx->workspace_bytes below what this call needs          */
   B2_STATUS_NOT_IMPLEMENTED = 3,
   B2_STATUS_TIMEOUT = 4,             /* only ever written to *ctx->device_status (trsv waits)    */
-  B2_STATUS_BAD_CONTEXT = 5          /* ctx NULL, workspace NULL / misaligned                    */
+  B2_STATUS_BAD_CONTEXT = 5,         /* ctx NULL, workspace NULL / misaligned                    */
+  B2_STATUS_TOO_LARGE = 6            /* problem size above the fixed limit of a *_noalloc call   */
 };
 
 /*
@@ -112,6 +113,25 @@ int b2_drot(const b2_ctx* ctx, int64_t n, double* x, int64_t incx, double* y, in
 /* dot: *result <- sum_i x_i*y_i.  Reductions are deterministic: same inputs, same bits. */
 int b2_sdot(const b2_ctx* ctx, int64_t n, const float* x, int64_t incx, const float* y, int64_t incy, float* result);
 int b2_ddot(const b2_ctx* ctx, int64_t n, const double* x, int64_t incx, const double* y, int64_t incy, double* result);
+
+/* sdot without any caller-provided or allocated scratch (the paper has no counterpart: this
+ * entry point exists for deployment reasons only).  Same result contract as b2_sdot, but no
+ * b2_ctx: the per-block partial sums and the ticket word sit in a fixed array inside the
+ * library's device image (4352 bytes; every GPU that loads the library carries it until the
+ * process exits).  It is meant for callers that cannot obtain device memory at the point of
+ * the call -- a plug-in running inside a host application whose allocator owns the whole GPU
+ * heap, a control loop whose rules forbid allocation after start-up because cudaMalloc may
+ * block and synchronise the device, a code path that runs after an out-of-memory condition.
+ * The entry point calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   stream   cudaStream_t to launch on (NULL = legacy default stream).
+ *   n        0 <= n <= 2^30; larger n returns B2_STATUS_TOO_LARGE and launches nothing.
+ *   others   as b2_sdot (device pointers, non-zero increments).
+ * The first call on each device looks up the device address of the array; make that first
+ * call outside any stream capture.  All calls share the one array: it still holds the last
+ * call's partials, the ticket word is cleared by every call before its kernel, and two calls
+ * that may overlap on the GPU (different streams, no ordering) race on it -- serialise them. */
+int b2_sdot_noalloc(void* stream, int64_t n, const float* x, int64_t incx, const float* y, int64_t incy,
+                    float* result);
 
 /* asum: *result <- sum_i |x_i|. */
 int b2_sasum(const b2_ctx* ctx, int64_t n, const float* x, int64_t incx, float* result);

@@ -23,6 +23,7 @@ NON_UNIT, UNIT = 131, 132
 
 STATUS_OK, STATUS_LAUNCH_FAILED, STATUS_WORKSPACE_TOO_SMALL = 0, 1, 2
 STATUS_NOT_IMPLEMENTED, STATUS_TIMEOUT, STATUS_BAD_CONTEXT = 3, 4, 5
+STATUS_TOO_LARGE = 6
 
 KNOB_L1_BLOCKS_PER_SM, KNOB_GEMV_N_TILE_BYTES, KNOB_GEMV_T_ROWS, KNOB_TRI_ROWS = 0, 1, 2, 3
 KNOB_GER_ROWS, KNOB_USE_PDL, KNOB_TRSV_DEBUG_SKIP, KNOB_TRI_WIDE = 4, 5, 6, 7
@@ -62,6 +63,7 @@ def _protos():
         out[f"b2_{p}symv"] = [cp, _int, _int, _i64, sc, _vp, _i64, _vp, _i64, sc, _vp, _i64]
         out[f"b2_{p}trmv"] = [cp, _int, _int, _int, _int, _i64, _vp, _i64, _vp, _i64]
         out[f"b2_{p}trsv"] = [cp, _int, _int, _int, _int, _i64, _vp, _i64, _vp, _i64]
+    out["b2_sdot_noalloc"] = [_vp, _i64, _vp, _i64, _vp, _i64, _vp]
     out["b2_workspace_reset"] = [cp]
     return out
 
@@ -227,3 +229,15 @@ def get_tuning(knob: int) -> int:
 
 def launch_count() -> int:
     return int(lib().b2_launch_count())
+
+
+def sdot_noalloc(n, x, incx, y, incy, result, stream=None, check=True):
+    """b2_sdot_noalloc: float dot product that needs no Context (no workspace): its scratch is a
+    fixed array inside the library.  For callers that cannot get device memory when they call;
+    calls must not overlap on the GPU."""
+    if stream is None:
+        stream = torch.cuda.current_stream(x.device).cuda_stream
+    st = lib().b2_sdot_noalloc(stream, n, _p(x), incx, _p(y), incy, _p(result))
+    if check and st != 0:
+        raise B2Error("b2_sdot_noalloc", st)
+    return st

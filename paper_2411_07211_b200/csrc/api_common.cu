@@ -52,6 +52,7 @@ const char* b2_status_string(int status) {
     case B2_STATUS_WORKSPACE_TOO_SMALL: return "workspace too small";
     case B2_STATUS_NOT_IMPLEMENTED: return "not implemented";
     case B2_STATUS_TIMEOUT: return "a bounded device-side wait ran out";
+    case B2_STATUS_TOO_LARGE: return "problem size above the fixed limit of this entry point";
     case B2_STATUS_BAD_CONTEXT: return "bad context (NULL, or workspace NULL / not 256-byte aligned)";
     default: return "unknown status";
   }

@@ -548,3 +548,69 @@ B2_L1_ONE_VEC_REDUCE(b2_isamax, float, IamaxOp, int64_t)
 B2_L1_ONE_VEC_REDUCE(b2_idamax, double, IamaxOp, int64_t)
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------- b2_sdot_noalloc
+// A dot product for callers that own no device scratch and may not allocate any.  The
+// partials and the ticket word that b2_sdot keeps in ctx->workspace live here in a fixed
+// file-scope device array instead.  Layout: word 0 = ticket, partials from byte 256 on.
+namespace b2 {
+constexpr int kNoAllocMaxBlocks = 1024;
+constexpr size_t kNoAllocScratchBytes = 256 + kNoAllocMaxBlocks * sizeof(float);
+constexpr int64_t kNoAllocMaxN = (int64_t)1 << 30;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+// In host code `g_noalloc_scratch` is only a handle: its device address has to be asked for,
+// once per device, with that device current.
+static int noalloc_scratch(unsigned char** out) {
+  static unsigned char* cached[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return B2_STATUS_LAUNCH_FAILED;
+  if (cached[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
+      (void)cudaGetLastError();
+      return B2_STATUS_LAUNCH_FAILED;
+    }
+    cached[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = cached[dev];
+  return B2_STATUS_OK;
+}
+}  // namespace b2
+
+extern "C" int b2_sdot_noalloc(void* stream, int64_t n, const float* x, int64_t incx, const float* y, int64_t incy,
+                               float* result) {
+  constexpr int XP = 2;
+  B2_L1_TWO_VEC_CHECK();
+  if (result == nullptr) return -6;
+  if (n > kNoAllocMaxN) return B2_STATUS_TOO_LARGE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (n == 0)
+    return cudaMemsetAsync(result, 0, sizeof(float), st) == cudaSuccess ? B2_STATUS_OK : B2_STATUS_LAUNCH_FAILED;
+  unsigned char* scratch = nullptr;
+  if (int rc = noalloc_scratch(&scratch)) return rc;
+  unsigned* ticket = reinterpret_cast<unsigned*>(scratch);
+  float* partials = reinterpret_cast<float*>(scratch + 256);
+  // The array keeps whatever the previous call left; the ticket must start at zero.
+  if (cudaMemsetAsync(ticket, 0, sizeof(unsigned), st) != cudaSuccess) return B2_STATUS_LAUNCH_FAILED;
+  using Op = DotOp<float>;
+  constexpr int V = VecLen<float>::value;
+  int64_t head = 0;
+  if (incx == 1 && incy == 1 && same_head<float>(x, y, true, &head)) {
+    constexpr int NV = 4;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) / V;
+    const int64_t nchunks = (nvec + kThreads * NV - 1) / (kThreads * NV);
+    const int64_t grid = nchunks < 1 ? 1 : (nchunks > kNoAllocMaxBlocks ? kNoAllocMaxBlocks : nchunks);
+    l1_reduce_unit<float, Op, NV><<<(unsigned)grid, kThreads, 0, st>>>(x, y, n, head, nvec, nchunks, partials, ticket,
+                                                                      result);
+  } else {
+    constexpr int NE = 8;
+    const int64_t nchunks = (n + kThreads * NE - 1) / (kThreads * NE);
+    const int64_t grid = nchunks > kNoAllocMaxBlocks ? kNoAllocMaxBlocks : nchunks;
+    l1_reduce_strided<float, Op, NE><<<(unsigned)grid, kThreads, 0, st>>>(vec_base(x, n, incx), incx,
+                                                                         vec_base(y, n, incy), incy, n, nchunks,
+                                                                         partials, ticket, result);
+  }
+  return check_launch();
+}
