@@ -382,6 +382,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--filter", default=None, help="only variants whose name contains one of these comma-separated "
+                                                   "strings (tuning runs; the headline run uses all)")
     ap.add_argument("--table", default=None, help="also write the per-variant table (JSON) to this path")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -402,6 +404,9 @@ def main():
 
     from paper_2411_07211_b200 import binding as b2
     wl = GpuWorkload(device)
+    if args.filter:
+        keys = args.filter.split(",")
+        wl.specs = [sp for sp in wl.specs if any(k in sp["name"] for k in keys)]
     nv = len(wl.specs)
     warm = max(3, args.warmup)
     for _ in range(warm):

@@ -12,6 +12,7 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobUsePdl          */ 1,
     /* kKnobTrsvDebugSkip   */ -1,
     /* kKnobTriWide         */ 0,
+    /* kKnobTrsvPrefetchBytes */ 48 << 20,
 };
 
 unsigned long long g_launch_count = 0;

@@ -153,6 +153,7 @@ enum Knob {
   kKnobUsePdl = 5,
   kKnobTrsvDebugSkip = 6,  // test hook: solve-order block that never publishes (-1 = none)
   kKnobTriWide = 7,
+  kKnobTrsvPrefetchBytes = 8,  // total L2 bytes trsv blocks may prefetch ahead of the front
   kKnobCount = 16
 };
 int64_t knob(int id);
