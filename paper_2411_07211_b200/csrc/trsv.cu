@@ -214,7 +214,10 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
   // 1a. diagonal block -> E (zero elsewhere, identity on unused / unit diagonal); b -> bvec
   for (int idx = tid; idx < kNB * kES; idx += kTT) E[idx] = T(0);
   for (int idx = tid; idx < kNB * kIS; idx += kTT) Einv[idx] = T(0);
-  if (tid < kNB) bvec[tid] = tid < nbI ? p.x[(r0 + solve_idx(tid)) * p.incx] : T(0);
+  if (tid < kNB) {
+    bvec[tid] = tid < nbI ? p.x[(r0 + solve_idx(tid)) * p.incx] : T(0);
+    racc[tid] = T(0);  // entries past a ragged block stay zero
+  }
   __syncthreads();
   for (int idx = tid; idx < kNB * kNB; idx += kTT) {
     const int pr = idx / kNB, pc = idx % kNB;  // position inside the stored block
