@@ -133,7 +133,7 @@ class ClockSampler:
 class GpuWorkload:
     """Device buffers (seeded synthetic data) and one launcher per variant."""
 
-    def __init__(self, device):
+    def __init__(self, device, name_filter=None):
         import torch
         from paper_2411_07211_b200 import binding as b2
         from paper_2411_07211_b200 import synth
@@ -142,10 +142,16 @@ class GpuWorkload:
         self.ctx = b2.Context(device)
         self.ctx.reset()
         self.specs = variant_specs()
+        if name_filter:
+            keys = name_filter.split(",")
+            self.specs = [sp for sp in self.specs if any(k in sp["name"] for k in keys)]
+        dtypes = {sp["dtype"] for sp in self.specs}
         self.flush = torch.empty(256 * MIB, dtype=torch.uint8, device=device)
         tdt = {"f32": torch.float32, "f64": torch.float64}
         self.buf = {}
         for dt, s in (("f32", 4), ("f64", 8)):
+            if dt not in dtypes:
+                continue
             t = tdt[dt]
             nel = 256 * MIB // s
             # level-1 vectors: X is a 256 MiB span, Y a 128 MiB span (+1 so inc=2 spans fit)
@@ -403,10 +409,7 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     from paper_2411_07211_b200 import binding as b2
-    wl = GpuWorkload(device)
-    if args.filter:
-        keys = args.filter.split(",")
-        wl.specs = [sp for sp in wl.specs if any(k in sp["name"] for k in keys)]
+    wl = GpuWorkload(device, args.filter)
     nv = len(wl.specs)
     warm = max(3, args.warmup)
     for _ in range(warm):

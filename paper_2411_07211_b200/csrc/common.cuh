@@ -70,6 +70,20 @@ __device__ __forceinline__ Pack<T, N> ld_nc(const T* p) {
   return r;
 }
 
+// Read-only load of reused data (the x vectors): cached in L1.
+template <typename T, int N>
+__device__ __forceinline__ Pack<T, N> ld_ro(const T* p) {
+  Pack<T, N> r;
+  if constexpr (sizeof(T) * N == 16) {
+    uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
+    r = *reinterpret_cast<Pack<T, N>*>(&t);
+  } else {
+    static_assert(N == 1, "packs are 16 bytes or one element");
+    r.v[0] = __ldg(p);
+  }
+  return r;
+}
+
 template <typename T, int N>
 __device__ __forceinline__ void st_cs(T* p, const Pack<T, N>& r) {
   if constexpr (sizeof(T) * N == 16) {
@@ -94,6 +108,31 @@ __device__ __forceinline__ T group_sum(T v) {
 #pragma unroll
   for (int m = LANES / 2; m >= 1; m >>= 1) v += shfl_xor(v, m);
   return v;
+}
+
+// Sums R values at once over each aligned group of LANES lanes (R a power of two <= LANES).
+// The first log2(R) butterfly steps trade half of the values for the partner's other half, so
+// the work shrinks with the lane span; plain butterflies finish the job.  Afterwards every
+// lane holds the total of value index (lane % LANES) / (LANES / R).  Fixed order.
+template <int LANES, int R, typename T>
+__device__ __forceinline__ T multi_group_sum(T (&v)[R], int lane) {
+  static_assert(R >= 1 && LANES >= R, "need at least one lane per value");
+  int span = LANES;
+#pragma unroll
+  for (int n = R; n > 1; n >>= 1) {
+    const int m = span >> 1, h = n >> 1;
+    const bool up = (lane & m) != 0;
+#pragma unroll
+    for (int i = 0; i < h; ++i) {
+      const T send = up ? v[i] : v[i + h];
+      const T keep = up ? v[i + h] : v[i];
+      v[i] = keep + shfl_xor(send, m);
+    }
+    span = m;
+  }
+#pragma unroll
+  for (int m = (LANES / R) >> 1; m >= 1; m >>= 1) v[0] += shfl_xor(v[0], m);
+  return v[0];
 }
 
 // Sum over the lanes that share (lane % LANES): the complementary butterfly.

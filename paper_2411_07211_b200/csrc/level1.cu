@@ -367,6 +367,19 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_strided(const T* __restric
 // ------------------------------------------------------------------------------- host side
 static int grid_cap() { return sm_count() * (int)knob(kKnobL1BlocksPerSm); }
 
+// One resident wave: as many blocks as really fit (the kernel grid-strides over the data), so
+// no second, partly filled wave trails behind.
+template <class Kernel>
+static int one_wave(Kernel kernel, int cap) {
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm <= 0) {
+    (void)cudaGetLastError();
+    return cap;
+  }
+  const int wave = per_sm * sm_count();
+  return wave < cap ? wave : cap;
+}
+
 template <typename T>
 static bool same_head(const T* x, const T* y, bool use_y, int64_t* head) {
   constexpr int V = VecLen<T>::value;
@@ -422,13 +435,15 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
     if (head > n) head = n;
     const int64_t nvec = (n - head) / V;
     const int64_t nchunks = (nvec + kThreads * NV - 1) / (kThreads * NV);
-    const int64_t grid = nchunks < 1 ? 1 : (nchunks > cap ? cap : nchunks);
+    static const int wave = one_wave(l1_reduce_unit<T, Op, NV>, cap);
+    const int64_t grid = nchunks < 1 ? 1 : (nchunks > wave ? wave : nchunks);
     l1_reduce_unit<T, Op, NV><<<(unsigned)grid, kThreads, 0, l.stream>>>(x, Op::RY ? y : x, n, head, nvec, nchunks,
                                                                         partials, ticket, result);
   } else {
     constexpr int NE = 8;
     const int64_t nchunks = (n + kThreads * NE - 1) / (kThreads * NE);
-    const int64_t grid = nchunks > cap ? cap : nchunks;
+    static const int wave = one_wave(l1_reduce_strided<T, Op, NE>, cap);
+    const int64_t grid = nchunks > wave ? wave : nchunks;
     l1_reduce_strided<T, Op, NE><<<(unsigned)grid, kThreads, 0, l.stream>>>(
         vec_base(x, n, incx), incx, Op::RY ? vec_base(y, n, incy) : x, Op::RY ? incy : 1, n, nchunks, partials, ticket,
         result);

@@ -54,6 +54,7 @@ struct L2Args {
   int64_t rows_per_cta;
   int ctiles_per_cta, nct, nrs, ncs;
   int direct;  // 1: blocks write alpha*acc + beta*y straight to y
+  int xc_vec;  // 1: xc has unit stride and 16-byte alignment, so it can be read in packs
   T alpha, beta;
   T* y;
   int64_t incy;
@@ -118,13 +119,22 @@ __global__ void __launch_bounds__(kThreads) l2_tile_kernel(const L2Args<T> p) {
       if (!region_active<K::TRI>(rb, rb_end, c0, c1)) continue;
       if (K::ROWOUT && xcv_ct != ct) {
         xcv_ct = ct;
+        if (V > 1 && p.xc_vec && c0 + TC <= p.cols) {
 #pragma unroll
-        for (int u = 0; u < CU; ++u)
+          for (int u = 0; u < CU; ++u) {
+            const P xv = ld_ro<T, V>(p.xc + c0 + (u * LPR + q) * V);
 #pragma unroll
-          for (int e = 0; e < V; ++e) {
-            const int64_t j = c0 + (u * LPR + q) * V + e;
-            xcv[u][e] = j < p.cols ? __ldg(p.xc + j * p.incxc) : T(0);
+            for (int e = 0; e < V; ++e) xcv[u][e] = xv.v[e];
           }
+        } else {
+#pragma unroll
+          for (int u = 0; u < CU; ++u)
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+              const int64_t j = c0 + (u * LPR + q) * V + e;
+              xcv[u][e] = j < p.cols ? __ldg(p.xc + j * p.incxc) : T(0);
+            }
+        }
       }
       const bool fast = (rb + RB <= r_end) && (c0 + TC <= p.cols) &&
                         region_strictly_inside<K::TRI>(rb, rb + RB, c0, c0 + TC);
@@ -176,18 +186,16 @@ __global__ void __launch_bounds__(kThreads) l2_tile_kernel(const L2Args<T> p) {
         }
       }
     }
-    if (K::ROWOUT) {
-#pragma unroll
-      for (int ru = 0; ru < RU; ++ru) {
-        const T s = group_sum<LPR>(rowacc[ru]);
-        const int64_t i = rowi[ru];
-        if (q == 0 && i < r_end) {
-          if (p.direct) {
-            T* yp = p.y + i * p.incy;
-            *yp = p.beta != T(0) ? p.alpha * s + p.beta * *yp : p.alpha * s;
-          } else {
-            p.rowpart[(int64_t)cs * p.rows + i] = s;
-          }
+    if (K::ROWOUT) {  // all RU row sums in one transposing butterfly
+      constexpr int LPV = LPR / RU;  // lanes left per row after the reduction
+      const T s = multi_group_sum<LPR, RU>(rowacc, lane);
+      const int64_t i = rb + ((q / LPV) * kWarps + warp) * G + g;
+      if (q % LPV == 0 && i < r_end) {
+        if (p.direct) {
+          T* yp = p.y + i * p.incy;
+          *yp = p.beta != T(0) ? p.alpha * s + p.beta * *yp : p.alpha * s;
+        } else {
+          p.rowpart[(int64_t)cs * p.rows + i] = s;
         }
       }
     }
@@ -301,6 +309,7 @@ static int l2_launch_shape(const Launch& l, L2Args<T> args, int64_t rows_per_cta
   constexpr int TC = S::template tc<V>();
   constexpr int RB = S::RB;
   args.nct = (int)((args.cols + TC - 1) / TC);
+  args.xc_vec = (K::ROWOUT && V > 1 && args.incxc == 1 && aligned_to(args.xc, 16)) ? 1 : 0;
   if (K::COLOUT) ctiles_per_cta = 1;
   if (ctiles_per_cta < 1) ctiles_per_cta = 1;
   if (ctiles_per_cta > args.nct) ctiles_per_cta = args.nct;
