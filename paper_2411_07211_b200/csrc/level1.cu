@@ -153,33 +153,51 @@ __global__ void __launch_bounds__(kThreads) l1_map_strided(Op op, T* __restrict_
 // ------------------------------------------------------------------------------- reduce ops
 template <typename T>
 struct DotOp {
+  static constexpr bool kArgmax = false;
+  static constexpr int kPacks = 4;  // 16-byte packs in flight per thread and array
   using Acc = T;
   using Out = T;
+  using Slot = T;  // per-thread running value of the streaming loop
+  __device__ __forceinline__ static Slot slot_init() { return T(0); }
+  __device__ __forceinline__ static Acc slot_to_acc(Slot s, int64_t, int64_t) { return s; }
   static constexpr bool RY = true;
   __device__ __forceinline__ static Acc init() { return T(0); }
   __device__ __forceinline__ static void accum(Acc& a, T x, T y, int64_t) { a = x * y + a; }
+  __device__ __forceinline__ static void slot_accum(Slot& a, T x, T y, int) { a = x * y + a; }
   __device__ __forceinline__ static Acc combine(Acc a, Acc b) { return a + b; }
   __device__ __forceinline__ static Acc shfl(Acc a, int m) { return shfl_xor(a, m); }
   __device__ __forceinline__ static Out finalize(Acc a) { return a; }
 };
 template <typename T>
 struct AsumOp {
+  static constexpr bool kArgmax = false;
+  static constexpr int kPacks = 8;  // 16-byte packs in flight per thread and array
   using Acc = T;
   using Out = T;
+  using Slot = T;  // per-thread running value of the streaming loop
+  __device__ __forceinline__ static Slot slot_init() { return T(0); }
+  __device__ __forceinline__ static Acc slot_to_acc(Slot s, int64_t, int64_t) { return s; }
   static constexpr bool RY = false;
   __device__ __forceinline__ static Acc init() { return T(0); }
   __device__ __forceinline__ static void accum(Acc& a, T x, T, int64_t) { a += fabs(x); }
+  __device__ __forceinline__ static void slot_accum(Slot& a, T x, T, int) { a += fabs(x); }
   __device__ __forceinline__ static Acc combine(Acc a, Acc b) { return a + b; }
   __device__ __forceinline__ static Acc shfl(Acc a, int m) { return shfl_xor(a, m); }
   __device__ __forceinline__ static Out finalize(Acc a) { return a; }
 };
 template <typename T>
 struct Nrm2Op {
+  static constexpr bool kArgmax = false;
+  static constexpr int kPacks = 8;  // 16-byte packs in flight per thread and array
   using Acc = T;
   using Out = T;
+  using Slot = T;  // per-thread running value of the streaming loop
+  __device__ __forceinline__ static Slot slot_init() { return T(0); }
+  __device__ __forceinline__ static Acc slot_to_acc(Slot s, int64_t, int64_t) { return s; }
   static constexpr bool RY = false;
   __device__ __forceinline__ static Acc init() { return T(0); }
   __device__ __forceinline__ static void accum(Acc& a, T x, T, int64_t) { a = x * x + a; }
+  __device__ __forceinline__ static void slot_accum(Slot& a, T x, T, int) { a = x * x + a; }
   __device__ __forceinline__ static Acc combine(Acc a, Acc b) { return a + b; }
   __device__ __forceinline__ static Acc shfl(Acc a, int m) { return shfl_xor(a, m); }
   __device__ __forceinline__ static Out finalize(Acc a) { return sqrt(a); }
@@ -193,6 +211,8 @@ struct MaxIdx {
 // larger magnitude, or on an equal magnitude with a smaller index.
 template <typename T>
 struct IamaxOp {
+  static constexpr int kPacks = 8;
+  static constexpr bool kArgmax = true;  // the kernels take the max-then-locate path
   using Acc = MaxIdx<T>;
   using Out = int64_t;
   static constexpr bool RY = false;
@@ -269,6 +289,10 @@ __device__ __forceinline__ void reduce_finish(typename Op::Acc acc, typename Op:
   }
 }
 
+// Streaming pass of the sum-type reductions: NV*V independent running values per thread.
+// The arg-max reduction (iamax) instead keeps ONE running maximum per thread: a max tree per
+// chunk costs about one instruction per element, and only when a chunk raises the maximum is
+// the first element that attains it located, while the chunk is still in registers.
 template <typename T, class Op, int NV>
 __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__ x, const T* __restrict__ y, int64_t n,
                                                            int64_t head, int64_t nvec, int64_t nchunks,
@@ -279,54 +303,93 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
   using Acc = typename Op::Acc;
   const T* xv = x + head;
   const T* yv = y + head;
-  Acc acc[NV][V];
-#pragma unroll
-  for (int k = 0; k < NV; ++k)
-#pragma unroll
-    for (int q = 0; q < V; ++q) acc[k][q] = Op::init();
-
-  for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
-    const int64_t v0 = chunk * (int64_t)(kThreads * NV) + threadIdx.x;
-    P px[NV], py[NV];
-    if (v0 + (int64_t)(NV - 1) * kThreads < nvec) {
-#pragma unroll
-      for (int k = 0; k < NV; ++k) {
-        const int64_t e = (v0 + (int64_t)k * kThreads) * V;
-        px[k] = ld_nc<T, V>(xv + e);
-        if (Op::RY) py[k] = ld_nc<T, V>(yv + e);
-      }
-#pragma unroll
-      for (int k = 0; k < NV; ++k) {
-        const int64_t e = head + (v0 + (int64_t)k * kThreads) * V;
-#pragma unroll
-        for (int q = 0; q < V; ++q) Op::accum(acc[k][q], px[k].v[q], Op::RY ? py[k].v[q] : T(0), e + q);
-      }
-    } else {
+  Acc a = Op::init();
+  if constexpr (Op::kArgmax) {
+    T best = T(-1);
+    int64_t best_chunk = -1;
+    int best_pos = 0;  // k*V + q inside that chunk
+    for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+      const int64_t v0 = chunk * (int64_t)(kThreads * NV) + threadIdx.x;
+      P px[NV];
+      T m = T(-1);
 #pragma unroll
       for (int k = 0; k < NV; ++k) {
         const int64_t v = v0 + (int64_t)k * kThreads;
-        if (v < nvec) {
-          px[k] = ld_nc<T, V>(xv + v * V);
-          if (Op::RY) py[k] = ld_nc<T, V>(yv + v * V);
+        if (v < nvec) px[k] = ld_nc<T, V>(xv + v * V);
+      }
 #pragma unroll
-          for (int q = 0; q < V; ++q) Op::accum(acc[k][q], px[k].v[q], Op::RY ? py[k].v[q] : T(0), head + v * V + q);
+      for (int k = 0; k < NV; ++k) {
+        const int64_t v = v0 + (int64_t)k * kThreads;
+#pragma unroll
+        for (int q = 0; q < V; ++q) {
+          px[k].v[q] = v < nvec ? fabs(px[k].v[q]) : T(-1);
+          m = fmax(m, px[k].v[q]);  // fmax drops NaN operands
+        }
+      }
+      if (m > best) {  // strict: the earliest chunk wins ties; locate while the data is in registers
+        best = m;
+        best_chunk = chunk;
+#pragma unroll
+        for (int k = NV - 1; k >= 0; --k)
+#pragma unroll
+          for (int q = V - 1; q >= 0; --q)
+            if (px[k].v[q] == m) best_pos = k * V + q;  // the lowest position is assigned last
+      }
+    }
+    if (best_chunk >= 0) {
+      const int k = best_pos / V, q = best_pos % V;
+      a = Acc{best, head + (best_chunk * (int64_t)(kThreads * NV) + threadIdx.x + (int64_t)k * kThreads) * V + q};
+    }
+  } else {
+    typename Op::Slot acc[NV][V];
+#pragma unroll
+    for (int k = 0; k < NV; ++k)
+#pragma unroll
+      for (int q = 0; q < V; ++q) acc[k][q] = Op::slot_init();
+    for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+      const int64_t v0 = chunk * (int64_t)(kThreads * NV) + threadIdx.x;
+      P px[NV], py[NV];
+      if (v0 + (int64_t)(NV - 1) * kThreads < nvec) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+          const int64_t e = (v0 + (int64_t)k * kThreads) * V;
+          px[k] = ld_nc<T, V>(xv + e);
+          if (Op::RY) py[k] = ld_nc<T, V>(yv + e);
+        }
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+          for (int q = 0; q < V; ++q) Op::slot_accum(acc[k][q], px[k].v[q], Op::RY ? py[k].v[q] : T(0), 0);
+      } else {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+          const int64_t v = v0 + (int64_t)k * kThreads;
+          if (v < nvec) {
+            px[k] = ld_nc<T, V>(xv + v * V);
+            if (Op::RY) py[k] = ld_nc<T, V>(yv + v * V);
+#pragma unroll
+            for (int q = 0; q < V; ++q) Op::slot_accum(acc[k][q], px[k].v[q], Op::RY ? py[k].v[q] : T(0), 0);
+          }
         }
       }
     }
+#pragma unroll
+    for (int k = 0; k < NV; ++k)
+#pragma unroll
+      for (int q = 0; q < V; ++q) a = Op::combine(a, Op::slot_to_acc(acc[k][q], 0, 0));
   }
-  Acc a = Op::init();
   if (blockIdx.x == 0) {  // scalar head and tail elements
     const int64_t tail0 = head + nvec * V;
     const int64_t ntail = n - tail0;
     int64_t i = -1;
     if ((int64_t)threadIdx.x < head) i = threadIdx.x;
     else if ((int64_t)threadIdx.x - head < ntail) i = tail0 + (threadIdx.x - head);
-    if (i >= 0) Op::accum(a, x[i], Op::RY ? y[i] : T(0), i);
+    if (i >= 0) {
+      Acc e = Op::init();
+      Op::accum(e, x[i], Op::RY ? y[i] : T(0), i);
+      a = Op::combine(a, e);
+    }
   }
-#pragma unroll
-  for (int k = 0; k < NV; ++k)
-#pragma unroll
-    for (int q = 0; q < V; ++q) a = Op::combine(a, acc[k][q]);
   reduce_finish<Op>(a, partials, ticket, result);
 }
 
@@ -336,31 +399,55 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_strided(const T* __restric
                                                               int64_t nchunks, typename Op::Acc* partials,
                                                               unsigned* ticket, typename Op::Out* result) {
   using Acc = typename Op::Acc;
-  Acc acc[NE];
+  Acc r = Op::init();
+  if constexpr (Op::kArgmax) {
+    T best = T(-1);
+    int64_t best_chunk = -1;
+    int best_pos = 0;
+    for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+      const int64_t i0 = chunk * (int64_t)(kThreads * NE) + threadIdx.x;
+      T a[NE];
 #pragma unroll
-  for (int k = 0; k < NE; ++k) acc[k] = Op::init();
-  for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
-    const int64_t i0 = chunk * (int64_t)(kThreads * NE) + threadIdx.x;
-    T a[NE], b[NE];
+      for (int k = 0; k < NE; ++k) {
+        const int64_t i = i0 + (int64_t)k * kThreads;
+        a[k] = i < n ? fabs(__ldg(x + i * incx)) : T(-1);
+      }
+      T m = T(-1);
 #pragma unroll
-    for (int k = 0; k < NE; ++k) {
-      const int64_t i = i0 + (int64_t)k * kThreads;
-      a[k] = T(0);
-      b[k] = T(0);
-      if (i < n) {
-        a[k] = __ldg(x + i * incx);
-        if (Op::RY) b[k] = __ldg(y + i * incy);
+      for (int k = 0; k < NE; ++k) m = fmax(m, a[k]);
+      if (m > best) {
+        best = m;
+        best_chunk = chunk;
+#pragma unroll
+        for (int k = NE - 1; k >= 0; --k)
+          if (a[k] == m) best_pos = k;
       }
     }
+    if (best_chunk >= 0) r = Acc{best, best_chunk * (int64_t)(kThreads * NE) + threadIdx.x + (int64_t)best_pos * kThreads};
+  } else {
+    typename Op::Slot acc[NE];
 #pragma unroll
-    for (int k = 0; k < NE; ++k) {
-      const int64_t i = i0 + (int64_t)k * kThreads;
-      if (i < n) Op::accum(acc[k], a[k], b[k], i);
+    for (int k = 0; k < NE; ++k) acc[k] = Op::slot_init();
+    for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+      const int64_t i0 = chunk * (int64_t)(kThreads * NE) + threadIdx.x;
+      T a[NE], b[NE];
+#pragma unroll
+      for (int k = 0; k < NE; ++k) {
+        const int64_t i = i0 + (int64_t)k * kThreads;
+        a[k] = T(0);
+        b[k] = T(0);
+        if (i < n) {
+          a[k] = __ldg(x + i * incx);
+          if (Op::RY) b[k] = __ldg(y + i * incy);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < NE; ++k)
+        if (i0 + (int64_t)k * kThreads < n) Op::slot_accum(acc[k], a[k], b[k], 0);
     }
-  }
-  Acc r = Op::init();
 #pragma unroll
-  for (int k = 0; k < NE; ++k) r = Op::combine(r, acc[k]);
+    for (int k = 0; k < NE; ++k) r = Op::combine(r, Op::slot_to_acc(acc[k], 0, 0));
+  }
   reduce_finish<Op>(r, partials, ticket, result);
 }
 
@@ -425,13 +512,14 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
                                                                                         : B2_STATUS_LAUNCH_FAILED;
   }
   constexpr int V = VecLen<T>::value;
+  if (n > ((int64_t)1 << 40)) return B2_STATUS_NOT_IMPLEMENTED;  // chunk ids are 32-bit
   const int cap = grid_cap();
   if (l.scratch_bytes < (size_t)cap * sizeof(Acc)) return B2_STATUS_WORKSPACE_TOO_SMALL;
   Acc* partials = reinterpret_cast<Acc*>(l.scratch);
   unsigned* ticket = l.ctl + kCtlReduceTicket;
   int64_t head = 0;
   if (incx == 1 && (!Op::RY || incy == 1) && same_head<T>(x, y, Op::RY, &head)) {
-    constexpr int NV = Op::RY ? 4 : 8;
+    constexpr int NV = Op::kPacks;
     if (head > n) head = n;
     const int64_t nvec = (n - head) / V;
     const int64_t nchunks = (nvec + kThreads * NV - 1) / (kThreads * NV);
@@ -440,7 +528,7 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
     l1_reduce_unit<T, Op, NV><<<(unsigned)grid, kThreads, 0, l.stream>>>(x, Op::RY ? y : x, n, head, nvec, nchunks,
                                                                         partials, ticket, result);
   } else {
-    constexpr int NE = 8;
+    constexpr int NE = Op::RY ? 8 : 16;
     const int64_t nchunks = (n + kThreads * NE - 1) / (kThreads * NE);
     static const int wave = one_wave(l1_reduce_strided<T, Op, NE>, cap);
     const int64_t grid = nchunks > wave ? wave : nchunks;
