@@ -1,38 +1,48 @@
 // trsv: solve op(A) x = b in place (Section 6.2.2; same option space as trmv).
 //
 // Blocked substitution with a dependency-ordered diagonal-block solve.  The unknowns are cut
-// into blocks of 64.  Thread blocks (512 threads) draw a ticket k = 0, 1, ... (the solve order: top-down for
-// an effectively lower-triangular op(A), bottom-up for an upper one); block k
-//   1. stages its 64x64 diagonal block in shared memory and inverts it there (recursive
-//      doubling, all threads) -- none of this depends on the solve,
-//   2. streams the off-diagonal tiles of its block row (or block column when op(A)'s rows are
-//      strided in memory) in solve order, two tiles per step, with the matrix data of the next
-//      step already in flight BEFORE it waits for the x values the current step multiplies,
-//   3. takes those x values from a side buffer in the workspace in which every value is
+// into blocks of 128; thread blocks draw a ticket k = 0, 1, ... (the solve order: top-down for
+// an effectively lower-triangular op(A), bottom-up for an upper one).  Block k
+//   1. stages its 128x128 diagonal block in shared memory and inverts it there, in place, by
+//      recursive doubling (none of this depends on the solve),
+//   2. streams the off-diagonal part of its block row (or block column when op(A)'s rows are
+//      strided in memory) as 128x64 tiles in solve order; 16 compute warps keep the next
+//      tile's matrix data in flight in registers and tiles further ahead are pulled into L2,
+//      all BEFORE the x values they multiply exist,
+//   3. receives those x values through a side buffer in the workspace in which every value is
 //      published as 64-bit words {32 payload bits, 32-bit call tag}: data and "ready" flag
-//      travel in one store, so a consumer polls the data itself (bounded; one warp polls for
-//      the block) and neither side needs a fence or a second round trip through L2,
-//   4. forms r = b - sum, multiplies by the inverted diagonal block (all threads), publishes
-//      its 64 values and writes them to the caller's x.
-// The chain of n/64 dependent steps makes the routine latency-bound; each step costs one
-// L2 store->load hand-over plus a 64x64 matvec.  Tickets are drawn in launch order, so a block
+//      travel in one store, so the consumer polls the data itself and neither side needs a
+//      fence or a second round trip through L2.  A 17th warp does nothing but poll (bounded)
+//      and hands decoded values to the compute warps through a ring of shared-memory buffers
+//      (named barriers), so polling latency never stalls the streaming warps, and only one warp
+//      per block loads the hot words -- a herd of pollers would swamp the L2 slice that
+//      holds them,
+//   4. forms r = b - sum, multiplies by the inverted diagonal block, publishes its 128 values
+//      and writes them to the caller's x.
+// The chain of n/128 dependent steps makes the routine latency-bound: each step costs one L2
+// store->load hand-over plus a 128x128 matvec.  Tickets are drawn in launch order, so a block
 // only ever waits for blocks that are already running: no co-residency assumption, no
-// deadlock.  If the polls of a thread exceed the iteration limit the block records
-// B2_STATUS_TIMEOUT in *device_status and leaves without publishing.
+// deadlock.  If the polls exceed the iteration limit the block records B2_STATUS_TIMEOUT in
+// *device_status and leaves without publishing (its dependants then time out too).
 //
 // Accuracy note: the diagonal blocks are applied through their explicit inverses (computed in
 // the working precision).  For diagonal blocks of moderate condition number this is as
-// accurate as substitution; it is the usual trade for removing 64 dependent steps per block.
+// accurate as substitution; it is the usual trade for removing 128 dependent steps per block.
 #include <atomic>
 
 #include "common.cuh"
 
 namespace b2 {
 
-constexpr int kNB = 64;
-constexpr int kTT = 512;          // threads per trsv block
-constexpr int kTW = kTT / 32;     // warps per trsv block
-constexpr int kGRP = 2;           // source tiles handled per loop iteration
+constexpr int kNB = 128;              // unknowns per thread block
+constexpr int kSB = 64;               // unknowns per source tile
+constexpr int kCW = 16;               // compute warps
+constexpr int kCT = kCW * 32;         // compute threads
+constexpr int kTT = kCT + 32;         // + one polling warp
+constexpr int kWS = kNB + 8;          // row stride of the diagonal-block array (16-byte row starts, conflict-free packs)
+constexpr int kXB = 4;                // x buffers between the polling warp and the compute warps
+constexpr int kBarFull = 1;           // named barriers kBarFull + b, kBarEmpty + b
+constexpr int kBarEmpty = 1 + kXB;
 
 __device__ __forceinline__ unsigned long long ld_word(const unsigned long long* p) {
   unsigned long long v;
@@ -41,6 +51,12 @@ __device__ __forceinline__ unsigned long long ld_word(const unsigned long long* 
 }
 __device__ __forceinline__ void st_word(unsigned long long* p, unsigned long long v) {
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void bar_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(int id, int count) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
 template <typename T>
@@ -51,7 +67,8 @@ struct TrsvArgs {
   int64_t incx;
   unsigned long long* xbuf;  // published solution: 1 (float) or 2 (double) tagged words per unknown
   unsigned* ticket;
-  int nb;
+  int nb;   // 128-blocks
+  int nsb;  // 64-blocks (source tiles)
   unsigned tag;
   unsigned long long wait_limit;
   int* device_status;
@@ -59,7 +76,7 @@ struct TrsvArgs {
   int pf_dist;  // L2 prefetch distance in tiles
 };
 
-// Per-thread polling state: a total budget of polls for the whole kernel.
+// Polling state of the polling warp's lanes: a total budget of polls for the whole kernel.
 struct Poller {
   unsigned long long budget;
   volatile int* abort_flag;  // shared memory
@@ -114,29 +131,30 @@ __device__ __forceinline__ double decode(const unsigned long long* w, double) {
 }
 
 // COLTYPE: op(A)'s rows are columns of the stored row-major view.  BACKWARD: solve bottom-up.
-constexpr int kES = kNB + 1;  // row stride of E   (conflict-free column walks)
-constexpr int kIS = kNB + 8;  // row stride of Einv (conflict-free for the 8-threads-per-row matvec)
-
 template <typename T, int V, bool COLTYPE, bool BACKWARD, bool UNIT>
 __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
-  constexpr int LPR = (kNB / V) >= 32 ? 32 : kNB / V;
-  constexpr int CU = kNB / (LPR * V);
+  // A tile is 128 own unknowns x 64 source unknowns; in memory it is 128 rows x 64 columns
+  // (rows of op(A) contiguous) or 64 rows x 128 columns (COLTYPE).
+  constexpr int TROWS = COLTYPE ? kSB : kNB, TCOLS = COLTYPE ? kNB : kSB;
+  constexpr int LPR = (TCOLS / V) >= 32 ? 32 : TCOLS / V;
+  constexpr int CU = TCOLS / (LPR * V);
   constexpr int G = 32 / LPR;
-  constexpr int RU = kNB / (kTW * G);
+  constexpr int RU = TROWS / (kCW * G);
   constexpr bool CANON_LOWER = (COLTYPE == BACKWARD);  // stored triangle in the row-major view
+  constexpr int WPE = Words<T>::N;
   using P = Pack<T, V>;
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  T* E = reinterpret_cast<T*>(smem_raw);  // diagonal block in solve order, E[s*kES + t], t <= s
-  T* Einv = E + kNB * kES;                // its inverse, Einv[s*kIS + t]
-  T* racc = Einv + kNB * kIS;             // sum over solved blocks, per unknown (solve order)
+  T* W = reinterpret_cast<T*>(smem_raw);  // diagonal block in solve order, W[s*kWS + t], then its inverse
+  T* racc = W + kNB * kWS;                // r = b - (sum over solved blocks), per unknown (solve order)
   T* bvec = racc + kNB;                   // right-hand side b (solve order)
-  T* xsm = bvec + kNB;                    // x values of the current tile group, double-buffered
-  T* colsm = xsm + 2 * kGRP * kNB;        // [kTW][kNB], COLTYPE only
+  T* xsm = bvec + kNB;                    // [kXB][kSB] x values handed over by the polling warp
+  T* colsm = xsm + kXB * kSB;             // [kCW][kNB], COLTYPE only
   __shared__ unsigned s_ticket;
   __shared__ int s_abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool poller = warp == kCW;
   const int g = lane / LPR, q = lane % LPR;
   if (tid == 0) {
     s_ticket = atomicAdd(p.ticket, 1u);
@@ -152,27 +170,20 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
   const int64_t r0 = (int64_t)I * kNB;
   const int nbI = (int)min((int64_t)kNB, p.n - r0);
   auto solve_idx = [&](int i) { return BACKWARD ? nbI - 1 - i : i; };
+  // source tiles (64 unknowns each) in solve order: s -> global 64-block index
+  const int nsrc = BACKWARD ? max(0, p.nsb - 2 * I - 2) : 2 * I;
+  auto src_block = [&](int s) { return BACKWARD ? p.nsb - 1 - s : s; };
 
   int lr[RU];
 #pragma unroll
-  for (int ru = 0; ru < RU; ++ru) lr[ru] = (ru * kTW + warp) * G + g;
+  for (int ru = 0; ru < RU; ++ru) lr[ru] = (ru * kCW + warp) * G + g;
 
   auto load_tile = [&](P (&av)[RU][CU], int s) {
-    if (s >= k) {  // padding tile of the last group
-#pragma unroll
-      for (int ru = 0; ru < RU; ++ru)
-#pragma unroll
-        for (int u = 0; u < CU; ++u)
-#pragma unroll
-          for (int e = 0; e < V; ++e) av[ru][u].v[e] = T(0);
-      return;
-    }
-    const int J = BACKWARD ? p.nb - 1 - s : s;
-    const int64_t c0 = (int64_t)J * kNB;
-    const int nbJ = (int)min((int64_t)kNB, p.n - c0);
+    const int64_t c0 = (int64_t)src_block(s) * kSB;
+    const int nbJ = (int)min((int64_t)kSB, p.n - c0);
     const int64_t rbase = COLTYPE ? c0 : r0, cbase = COLTYPE ? r0 : c0;
     const int nr = COLTYPE ? nbJ : nbI, nc = COLTYPE ? nbI : nbJ;
-    if (nr == kNB && nc == kNB) {
+    if (nr == TROWS && nc == TCOLS) {
 #pragma unroll
       for (int ru = 0; ru < RU; ++ru)
 #pragma unroll
@@ -189,84 +200,160 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
           }
     }
   };
-
   // Tiles further ahead are pulled into L2 while the block waits for the solve front, so DRAM
   // streams continuously instead of in bursts locked to the front (one 128-byte line per thread).
   auto prefetch_tile = [&](int s) {
-    if (s >= k) return;
-    const int J = BACKWARD ? p.nb - 1 - s : s;
-    const int64_t c0 = (int64_t)J * kNB;
-    if (p.n - c0 < kNB || nbI < kNB) return;  // ragged tiles are not worth it
+    if (s >= nsrc) return;
+    const int64_t c0 = (int64_t)src_block(s) * kSB;
+    if (p.n - c0 < kSB || nbI < kNB) return;  // ragged tiles are not worth it
     const int64_t rbase = COLTYPE ? c0 : r0, cbase = COLTYPE ? r0 : c0;
-    constexpr int LINES = kNB * (int)sizeof(T) / 128;
-    if (tid < kNB * LINES) {
-      const T* ptr = p.a + (rbase + tid / LINES) * p.lda + cbase + (tid % LINES) * (128 / (int)sizeof(T));
+    constexpr int LINES = TCOLS * (int)sizeof(T) / 128;
+    for (int i = tid; i < TROWS * LINES; i += kCT) {
+      const T* ptr = p.a + (rbase + i / LINES) * p.lda + cbase + (i % LINES) * (128 / (int)sizeof(T));
       asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
     }
   };
 
-  // The first tiles' matrix data go in flight before anything else.
-  P cur[kGRP][RU][CU], nxt[kGRP][RU][CU];
-#pragma unroll
-  for (int t = 0; t < kGRP; ++t) load_tile(nxt[t], t);
-  for (int s = kGRP; s < kGRP + p.pf_dist; ++s) prefetch_tile(s);
+  // The first tile's matrix data goes in flight before anything else.
+  P cur[RU][CU], nxt[RU][CU];
+  if (!poller) {
+    if (nsrc > 0) load_tile(nxt, 0);
+    for (int s = 1; s < 1 + p.pf_dist; ++s) prefetch_tile(s);
+  }
 
-  // 1a. diagonal block -> E (zero elsewhere, identity on unused / unit diagonal); b -> bvec
-  for (int idx = tid; idx < kNB * kES; idx += kTT) E[idx] = T(0);
-  for (int idx = tid; idx < kNB * kIS; idx += kTT) Einv[idx] = T(0);
+  // 1a. diagonal block -> W (zero elsewhere, identity on unused / unit diagonal); b -> bvec
+  for (int idx = tid; idx < kNB * kWS; idx += kTT) W[idx] = T(0);
   if (tid < kNB) {
     bvec[tid] = tid < nbI ? p.x[(r0 + solve_idx(tid)) * p.incx] : T(0);
-    racc[tid] = T(0);  // entries past a ragged block stay zero
+    racc[tid] = bvec[tid];  // r = b when nothing precedes; entries past a ragged block stay zero
   }
   __syncthreads();
-  for (int idx = tid; idx < kNB * kNB; idx += kTT) {
-    const int pr = idx / kNB, pc = idx % kNB;  // position inside the stored block
-    if (pr < nbI && pc < nbI) {
-      const bool in_tri = CANON_LOWER ? (pc <= pr) : (pc >= pr);
-      if (in_tri && !(UNIT && pr == pc)) {
-        const T v = __ldg(p.a + (r0 + pr) * p.lda + r0 + pc);
+  for (int base = 0; base < kNB * kNB; base += 8 * kTT) {  // 8 independent loads in flight per thread
+    T v[8];
+    bool use[8];
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      const int idx = base + m * kTT + tid;
+      const int pr = idx / kNB, pc = idx % kNB;  // position inside the stored block
+      use[m] = idx < kNB * kNB && pr < nbI && pc < nbI && (CANON_LOWER ? (pc <= pr) : (pc >= pr)) &&
+               !(UNIT && pr == pc);
+      v[m] = use[m] ? __ldg(p.a + (r0 + pr) * p.lda + r0 + pc) : T(0);
+    }
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      const int idx = base + m * kTT + tid;
+      const int pr = idx / kNB, pc = idx % kNB;
+      if (use[m]) {
         const int sr = solve_idx(pr), sc = solve_idx(pc);
-        if (COLTYPE) E[sc * kES + sr] = v;
-        else E[sr * kES + sc] = v;
+        if (COLTYPE) W[sc * kWS + sr] = v[m];
+        else W[sr * kWS + sc] = v[m];
       }
     }
   }
   for (int s = tid; s < kNB; s += kTT)
-    if (UNIT || s >= nbI) E[s * kES + s] = T(1);
+    if (UNIT || s >= nbI) W[s * kWS + s] = T(1);
   __syncthreads();
 
-  // 1b. inverse of E by recursive doubling.  8x8 diagonal blocks are inverted by substitution
-  // (one column per thread); then, for h = 8, 16, 32, every pair [A 0; C B] of h x h blocks gets
-  // its lower-left block  -B^-1 (C A^-1).  The intermediate C A^-1 is parked in the unused
-  // upper triangle of E (transposed position).
-  if (tid < kNB) {
-    const int c = tid, d0 = (c / 8) * 8;
-    for (int s = c; s < d0 + 8; ++s) {
-      T acc = (s == c) ? T(1) : T(0);
-      for (int t = c; t < s; ++t) acc -= E[s * kES + t] * Einv[t * kIS + c];
-      Einv[s * kIS + c] = acc / E[s * kES + s];
+  // 1b. in-place inverse by recursive doubling.  4x4 diagonal blocks: one column per thread,
+  // block held in registers, substitution on e_c.  Then, for h = 4 .. 64, every pair
+  // [A 0; C B] of h x h blocks gets its lower-left block -B^-1 (C A^-1); the intermediate
+  // C A^-1 is parked in the (unused) upper triangle at the transposed position.
+  {
+    T col[4];
+    const int c = tid, d0 = (c / 4) * 4, lc = c % 4;
+    if (tid < kNB) {
+      T e[4][4];
+#pragma unroll
+      for (int ls = 0; ls < 4; ++ls)
+#pragma unroll
+        for (int lt = 0; lt <= ls; ++lt) e[ls][lt] = W[(d0 + ls) * kWS + d0 + lt];
+#pragma unroll
+      for (int ls = 0; ls < 4; ++ls) {
+        T acc = (ls == lc) ? T(1) : T(0);
+#pragma unroll
+        for (int lt = 0; lt < ls; ++lt) acc -= e[ls][lt] * col[lt];
+        col[ls] = acc / e[ls][ls];
+      }
     }
+    __syncthreads();
+    if (tid < kNB) {
+#pragma unroll
+      for (int ls = 0; ls < 4; ++ls) W[(d0 + ls) * kWS + c] = col[ls];  // zero above the diagonal
+    }
+    __syncthreads();
   }
-  __syncthreads();
 #pragma unroll 1
-  for (int h = 8; h < kNB; h *= 2) {
-    const int per_pair = h * h, total = (kNB / (2 * h)) * per_pair;
-    for (int e = tid; e < total; e += kTT) {  // Tm = C * A^-1
-      const int pr = e / per_pair, i = (e % per_pair) / h, j = e % h;
+  for (int h = 4; h < kNB; h *= 2) {  // 4x4 register tiles: 8 shared-memory loads per 16 multiply-adds
+    const int tpr = h / 4, per_pair = tpr * tpr, total = (kNB / (2 * h)) * per_pair;
+    for (int e = tid; e < total; e += kTT) {  // Tm = C * A^-1  (A^-1 is zero above its diagonal)
+      const int pr = e / per_pair, i0 = ((e % per_pair) / tpr) * 4, j0 = (e % tpr) * 4;
       const int top = pr * 2 * h, bot = top + h;
-      T acc = T(0);
-      for (int l = j; l < h; ++l) acc = E[(bot + i) * kES + top + l] * Einv[(top + l) * kIS + top + j] + acc;
-      E[(top + j) * kES + bot + i] = acc;
+      T acc[4][4];
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) acc[ii][jj] = T(0);
+#pragma unroll 4
+      for (int l = j0; l < h; ++l) {
+        T cv[4], av[4];
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii) cv[ii] = W[(bot + i0 + ii) * kWS + top + l];
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) av[jj] = W[(top + l) * kWS + top + j0 + jj];
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) acc[ii][jj] = cv[ii] * av[jj] + acc[ii][jj];
+      }
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) W[(top + j0 + jj) * kWS + bot + i0 + ii] = acc[ii][jj];
     }
     __syncthreads();
-    for (int e = tid; e < total; e += kTT) {  // X = -B^-1 * Tm
-      const int pr = e / per_pair, i = (e % per_pair) / h, j = e % h;
+    for (int e = tid; e < total; e += kTT) {  // X = -B^-1 * Tm, written over C (B^-1 zero above its diagonal)
+      const int pr = e / per_pair, i0 = ((e % per_pair) / tpr) * 4, j0 = (e % tpr) * 4;
       const int top = pr * 2 * h, bot = top + h;
-      T acc = T(0);
-      for (int l = 0; l <= i; ++l) acc = Einv[(bot + i) * kIS + bot + l] * E[(top + j) * kES + bot + l] + acc;
-      Einv[(bot + i) * kIS + top + j] = -acc;
+      T acc[4][4];
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) acc[ii][jj] = T(0);
+#pragma unroll 4
+      for (int l = 0; l < i0 + 4; ++l) {
+        T bv[4], tv[4];
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii) bv[ii] = W[(bot + i0 + ii) * kWS + bot + l];
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) tv[jj] = W[(top + j0 + jj) * kWS + bot + l];
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) acc[ii][jj] = bv[ii] * tv[jj] + acc[ii][jj];
+      }
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) W[(bot + i0 + ii) * kWS + top + j0 + jj] = -acc[ii][jj];
     }
     __syncthreads();
+    for (int e = tid; e < (kNB / (2 * h)) * h * h; e += kTT) {  // scrub the parked intermediates
+      const int pr = e / (h * h), i = (e % (h * h)) / h, j = e % h;
+      W[(pr * 2 * h + j) * kWS + pr * 2 * h + h + i] = T(0);
+    }
+    __syncthreads();
+  }
+  // The finished inverse: float blocks keep their share in registers (the 128x128 matvec is then
+  // free of shared-memory traffic), double blocks read it from shared memory in 16-byte packs.
+  constexpr int VL = 16 / (int)sizeof(T);          // elements per pack
+  constexpr int TPU = kCT / kNB;                   // threads per unknown (4)
+  constexpr int NPK = kNB / (TPU * VL);            // packs per thread
+  constexpr bool WREG = sizeof(T) == 4;
+  Pack<T, VL> wreg[WREG ? NPK : 1];
+  if (WREG && !poller) {
+    const int ms = tid / TPU, part = tid % TPU;
+#pragma unroll
+    for (int m = 0; m < NPK; ++m) wreg[m] = *reinterpret_cast<const Pack<T, VL>*>(&W[ms * kWS + VL * (part + TPU * m)]);
   }
 
   // 2./3. off-diagonal tiles in solve order
@@ -279,121 +366,134 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
 #pragma unroll
     for (int e = 0; e < V; ++e) colacc[u][e] = T(0);
 
-  Poller poll;
-  poll.budget = p.wait_limit ? p.wait_limit : (1ull << 20);
-  poll.abort_flag = &s_abort;
-  poll.device_status = p.device_status;
-  poll.tag = p.tag;
-
-  // Tiles are taken kGRP at a time: one poll round trip and one loop iteration then serve
-  // kGRP tiles, which keeps a block with a long row ahead of the solve front.  The matrix data
-  // of the next group is already in flight while this group's x values are awaited.
-  constexpr int WPE = Words<T>::N;
-  const int ngroups = (k + kGRP - 1) / kGRP;
-#pragma unroll 1
-  for (int gi = 0; gi < ngroups; ++gi) {
-    const int s0 = gi * kGRP;
-#pragma unroll
-    for (int t = 0; t < kGRP; ++t)
-#pragma unroll
-      for (int ru = 0; ru < RU; ++ru)
-#pragma unroll
-        for (int u = 0; u < CU; ++u) cur[t][ru][u] = nxt[t][ru][u];
-    if (gi + 1 < ngroups) {
-#pragma unroll
-      for (int t = 0; t < kGRP; ++t) load_tile(nxt[t], s0 + kGRP + t);
-#pragma unroll
-      for (int t = 0; t < kGRP; ++t) prefetch_tile(s0 + kGRP + p.pf_dist + t);
-    }
-    // Warp 0 polls the group's tagged words on behalf of the block (one reader per block keeps
-    // the L2 slice that holds the front's words from being swamped) and hands the decoded
-    // values over through shared memory.  Blocks further from the front sleep between polls.
-    T* xg = xsm + (gi & 1) * (kGRP * kNB);
-    if (warp == 0) {
-      const int dist = k - min(k - 1, s0 + kGRP - 1);
+  if (poller) {
+    Poller poll;
+    poll.budget = p.wait_limit ? p.wait_limit : (1ull << 20);
+    poll.abort_flag = &s_abort;
+    poll.device_status = p.device_status;
+    poll.tag = p.tag;
+    // A solved block publishes 128 unknowns = two source tiles at once, so the tiles are polled
+    // in pairs: one round trip through L2 serves both.
+    constexpr int EPL = 2 * kSB / 32;  // unknowns per lane and pair
+    for (int s = 0; s < nsrc; s += 2) {
+      const int b0 = s % kXB, b1 = (s + 1) % kXB;
+      if (s >= kXB) bar_sync(kBarEmpty + b0, kTT);  // the compute warps are done with these buffers
+      if (s + 1 < nsrc && s + 1 >= kXB) bar_sync(kBarEmpty + b1, kTT);
+      // blocks further from the front sleep between polls so that only the next in line spins
+      const int last = min(s + 1, nsrc - 1);
+      const int dist = k - (BACKWARD ? p.nb - 1 - src_block(last) / 2 : src_block(last) / 2);
       poll.backoff_ns = dist > 1 ? (unsigned)min(dist - 1, 64) * 500u : 0u;
-      constexpr int EPL = kGRP * kNB / 32;  // unknowns per lane
       unsigned long long w[EPL * WPE];
       const unsigned long long* wp[EPL * WPE];
 #pragma unroll
       for (int j = 0; j < EPL; ++j) {
-        const int el = lane * EPL + j, t = el / kNB, lc = el % kNB;
-        const int s = s0 + t;
-        const int J = BACKWARD ? p.nb - 1 - s : s;
-        const int64_t c0 = (int64_t)J * kNB;
-        const bool valid = s < k && c0 + lc < p.n;
+        const int el = lane * EPL + j, t = el / kSB, lc = el % kSB;  // tile of the pair, position in it
+        const int64_t u = (int64_t)src_block(min(s + t, nsrc - 1)) * kSB + lc;
+        const bool valid = s + t < nsrc && u < p.n;
 #pragma unroll
-        for (int h = 0; h < WPE; ++h) wp[j * WPE + h] = valid ? p.xbuf + (c0 + lc) * WPE + h : nullptr;
+        for (int h = 0; h < WPE; ++h) wp[j * WPE + h] = valid ? p.xbuf + u * WPE + h : nullptr;
       }
       poll.wait_words(w, wp);
 #pragma unroll
-      for (int j = 0; j < EPL; ++j) xg[lane * EPL + j] = wp[j * WPE] ? decode(&w[j * WPE], T(0)) : T(0);
+      for (int j = 0; j < EPL; ++j) {
+        const int el = lane * EPL + j, t = el / kSB, lc = el % kSB;
+        xsm[(t ? b1 : b0) * kSB + lc] = wp[j * WPE] ? decode(&w[j * WPE], T(0)) : T(0);
+      }
+      __threadfence_block();
+      bar_arrive(kBarFull + b0, kTT);
+      if (s + 1 < nsrc) bar_arrive(kBarFull + b1, kTT);
     }
-    __syncthreads();
+  } else {
+#pragma unroll 1
+    for (int s = 0; s < nsrc; ++s) {
+      const int b = s % kXB;
 #pragma unroll
-    for (int t = 0; t < kGRP; ++t) {
+      for (int ru = 0; ru < RU; ++ru)
+#pragma unroll
+        for (int u = 0; u < CU; ++u) cur[ru][u] = nxt[ru][u];
+      if (s + 1 < nsrc) {
+        load_tile(nxt, s + 1);
+        prefetch_tile(s + 1 + p.pf_dist);
+      }
+      bar_sync(kBarFull + b, kTT);  // x values of this tile are in xsm[b]
+      const T* xg = xsm + b * kSB;
       if (COLTYPE) {
         T xr[RU];
 #pragma unroll
-        for (int ru = 0; ru < RU; ++ru) xr[ru] = xg[t * kNB + lr[ru]];
+        for (int ru = 0; ru < RU; ++ru) xr[ru] = xg[lr[ru]];
 #pragma unroll
         for (int ru = 0; ru < RU; ++ru)
 #pragma unroll
           for (int u = 0; u < CU; ++u)
 #pragma unroll
-            for (int e = 0; e < V; ++e) colacc[u][e] = cur[t][ru][u].v[e] * xr[ru] + colacc[u][e];
+            for (int e = 0; e < V; ++e) colacc[u][e] = cur[ru][u].v[e] * xr[ru] + colacc[u][e];
       } else {
         T xs[CU][V];
 #pragma unroll
         for (int u = 0; u < CU; ++u)
 #pragma unroll
-          for (int e = 0; e < V; ++e) xs[u][e] = xg[t * kNB + (u * LPR + q) * V + e];
+          for (int e = 0; e < V; ++e) xs[u][e] = xg[(u * LPR + q) * V + e];
 #pragma unroll
         for (int ru = 0; ru < RU; ++ru)
 #pragma unroll
           for (int u = 0; u < CU; ++u)
 #pragma unroll
-            for (int e = 0; e < V; ++e) rowacc[ru] = cur[t][ru][u].v[e] * xs[u][e] + rowacc[ru];
+            for (int e = 0; e < V; ++e) rowacc[ru] = cur[ru][u].v[e] * xs[u][e] + rowacc[ru];
       }
+      if (s + kXB < nsrc) bar_arrive(kBarEmpty + b, kTT);  // only if the polling warp will wait for it
     }
-  }
 
-  // per-unknown sums -> racc (solve order)
-  if (COLTYPE) {
+    // per-unknown sums -> racc (solve order)
+    if (COLTYPE) {
 #pragma unroll
-    for (int u = 0; u < CU; ++u)
+      for (int u = 0; u < CU; ++u)
 #pragma unroll
-      for (int e = 0; e < V; ++e) {
-        const T s = cross_group_sum<LPR>(colacc[u][e]);
-        if (g == 0) colsm[warp * kNB + (u * LPR + q) * V + e] = s;
-      }
-    __syncthreads();
-    if (tid < kNB) {
-      T s = colsm[tid];
-#pragma unroll
-      for (int w = 1; w < kTW; ++w) s += colsm[w * kNB + tid];
-      if (tid < nbI) racc[solve_idx(tid)] = s;
-    }
-  } else {
-#pragma unroll
-    for (int ru = 0; ru < RU; ++ru) {
-      const T s = group_sum<LPR>(rowacc[ru]);
-      if (q == 0 && lr[ru] < nbI) racc[solve_idx(lr[ru])] = s;
+        for (int e = 0; e < V; ++e) {
+          const T s = cross_group_sum<LPR>(colacc[u][e]);
+          if (g == 0) colsm[warp * kNB + (u * LPR + q) * V + e] = s;
+        }
+    } else {
+      constexpr int LPV = LPR / RU;  // lanes left per row after the reduction
+      const T s = multi_group_sum<LPR, RU>(rowacc, lane);
+      const int i = ((q / LPV) * kCW + warp) * G + g;
+      if (q % LPV == 0 && i < nbI) racc[solve_idx(i)] = bvec[solve_idx(i)] - s;
     }
   }
   __syncthreads();
+  if (COLTYPE) {
+    if (tid < nbI) {
+      T s = colsm[tid];
+#pragma unroll
+      for (int w = 1; w < kCW; ++w) s += colsm[w * kNB + tid];
+      racc[solve_idx(tid)] = bvec[solve_idx(tid)] - s;
+    }
+    __syncthreads();
+  }
   if (s_abort) return;  // a wait ran out: publish nothing, dependants will time out too
 
-  // 4. x = Einv * (b - racc): kTT/64 threads per unknown, then publish and write back
-  {
-    constexpr int TPU = kTT / kNB;  // threads per unknown (8)
+  // 4. x = W * r: 4 threads per unknown, then publish and write back
+  if (!poller) {
     const int s = tid / TPU, part = tid % TPU;
-    T acc = T(0);
+    T accv[VL];  // independent chains
 #pragma unroll
-    for (int j = 0; j < kNB / TPU; ++j) {
-      const int t = part + TPU * j;
-      acc = Einv[s * kIS + t] * (bvec[t] - racc[t]) + acc;  // Einv is zero above the diagonal
+    for (int e = 0; e < VL; ++e) accv[e] = T(0);
+#pragma unroll
+    for (int m = 0; m < NPK; ++m) {
+      const int t0 = VL * (part + TPU * m);
+      if (WREG) {
+        const Pack<T, VL> rv = *reinterpret_cast<const Pack<T, VL>*>(&racc[t0]);
+#pragma unroll
+        for (int e = 0; e < VL; ++e) accv[e] = wreg[m].v[e] * rv.v[e] + accv[e];
+      } else if (t0 <= s) {  // W is zero above the diagonal
+        const Pack<T, VL> wv = *reinterpret_cast<const Pack<T, VL>*>(&W[s * kWS + t0]);
+        const Pack<T, VL> rv = *reinterpret_cast<const Pack<T, VL>*>(&racc[t0]);
+#pragma unroll
+        for (int e = 0; e < VL; ++e) accv[e] = wv.v[e] * rv.v[e] + accv[e];
+      }
     }
+    T acc = accv[0];
+#pragma unroll
+    for (int e = 1; e < VL; ++e) acc += accv[e];
 #pragma unroll
     for (int m = 1; m < TPU; m <<= 1) acc += shfl_xor(acc, m);
     if (part == 0 && s < nbI && k != p.debug_skip) {
@@ -407,7 +507,7 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
 
 template <typename T, bool COLTYPE>
 constexpr size_t trsv_smem_bytes() {
-  return sizeof(T) * (kNB * kES + kNB * kIS + 2 * kNB + 2 * kGRP * kNB + (COLTYPE ? kTW : 1) * kNB);
+  return sizeof(T) * (kNB * kWS + 2 * kNB + kXB * kSB + (COLTYPE ? kCW : 0) * kNB);
 }
 
 template <typename T, int V, bool COLTYPE, bool BACKWARD, bool UNIT>
@@ -471,12 +571,13 @@ static int trsv_impl(const b2_ctx* ctx, int order, int uplo, int trans, int diag
   args.xbuf = reinterpret_cast<unsigned long long*>(l.scratch);
   args.ticket = l.ctl + kCtlTrsvTicket;
   args.nb = (int)((n + kNB - 1) / kNB);
+  args.nsb = (int)((n + kSB - 1) / kSB);
   args.tag = next_tag();
   args.wait_limit = l.wait_limit;
   args.device_status = l.device_status;
   args.debug_skip = (int)knob(kKnobTrsvDebugSkip);
   {  // keep the prefetched-but-unused tiles of all blocks within a fraction of L2
-    const int64_t tile_bytes = (int64_t)kNB * kNB * sizeof(T);
+    const int64_t tile_bytes = (int64_t)kNB * kSB * sizeof(T);
     int64_t d = knob(kKnobTrsvPrefetchBytes) / (tile_bytes * args.nb);
     args.pf_dist = (int)(d < 0 ? 0 : d > 64 ? 64 : d);
   }

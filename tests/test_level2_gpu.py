@@ -185,7 +185,7 @@ def test_trsv_bounded_wait_reports_timeout(b2):
     library), so its dependants' waits run out.  They must return a status, not hang."""
     ctx = b2.Context(wait_limit=2000)
     ctx.reset()
-    n = 64 * 6
+    n = 128 * 6
     a = Guarded(tri_buf(3, n, n, np.float32, orc.ROW_MAJOR, orc.LOWER, orc.NON_UNIT))
     x = Guarded(synth.vector_np(1, 1, n, np.float32))
     b2.set_tuning(b2.KNOB_TRSV_DEBUG_SKIP, 2)
