@@ -77,7 +77,7 @@ __device__ __forceinline__ bool region_strictly_inside(int64_t r0, int64_t r1, i
 }
 
 template <typename T, int V, class K, class S>
-__global__ void __launch_bounds__(kThreads) l2_tile_kernel(const L2Args<T> p) {
+__global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p) {
   constexpr int LPR = S::LPR, CU = S::CU, RU = S::RU, G = S::G, RB = S::RB;
   constexpr int TC = LPR * V * CU;
   using P = Pack<T, V>;
@@ -102,17 +102,29 @@ __global__ void __launch_bounds__(kThreads) l2_tile_kernel(const L2Args<T> p) {
     for (int e = 0; e < V; ++e) colacc[u][e] = T(0), xcv[u][e] = T(0);
   int xcv_ct = -1;  // column tile whose x values are in xcv
 
+  // Address arithmetic is hoisted: inside a tile everything is a 32-bit local index or a
+  // pointer bumped by a precomputed stride.
+  const int lrow0 = warp * G + g;                            // first local row of this thread
+  const int64_t rstride = (int64_t)kWarps * G * p.lda;       // elements between a thread's rows
+  const int64_t xstride = (int64_t)kWarps * G * p.incxr;
+  const T* a_cta = p.a + (r_begin + lrow0) * p.lda + q * V;  // row r_begin + lrow0, column q*V
+
   for (int64_t rb = r_begin; rb < r_end; rb += RB) {
     const int64_t rb_end = min(rb + RB, r_end);
     if (!region_active<K::TRI>(rb, rb_end, c_lo, c_hi)) continue;
+    const int nr = (int)(rb_end - rb);  // rows of this batch
+    const T* a_rb = a_cta + (rb - r_begin) * p.lda;
     T rowacc[RU], xrv[RU];
-    int64_t rowi[RU];
 #pragma unroll
     for (int ru = 0; ru < RU; ++ru) {
-      rowi[ru] = rb + (ru * kWarps + warp) * G + g;
       rowacc[ru] = T(0);
       xrv[ru] = T(0);
-      if (K::COLOUT && rowi[ru] < r_end) xrv[ru] = __ldg(p.xr + rowi[ru] * p.incxr);
+    }
+    if (K::COLOUT) {
+      const T* xp = p.xr + (rb + lrow0) * p.incxr;
+#pragma unroll
+      for (int ru = 0; ru < RU; ++ru)
+        if (lrow0 + ru * kWarps * G < nr) xrv[ru] = __ldg(xp + ru * xstride);
     }
     for (int ct = ct_begin; ct < ct_end; ++ct) {
       const int64_t c0 = (int64_t)ct * TC, c1 = min(p.cols, c0 + TC);
@@ -140,10 +152,11 @@ __global__ void __launch_bounds__(kThreads) l2_tile_kernel(const L2Args<T> p) {
                         region_strictly_inside<K::TRI>(rb, rb + RB, c0, c0 + TC);
       if (fast) {
         P av[RU][CU];
+        const T* at = a_rb + c0;
 #pragma unroll
         for (int ru = 0; ru < RU; ++ru)
 #pragma unroll
-          for (int u = 0; u < CU; ++u) av[ru][u] = ld_nc<T, V>(p.a + rowi[ru] * p.lda + c0 + (u * LPR + q) * V);
+          for (int u = 0; u < CU; ++u) av[ru][u] = ld_nc<T, V>(at + ru * rstride + u * (LPR * V));
 #pragma unroll
         for (int ru = 0; ru < RU; ++ru)
 #pragma unroll
@@ -154,30 +167,37 @@ __global__ void __launch_bounds__(kThreads) l2_tile_kernel(const L2Args<T> p) {
               if (K::COLOUT) colacc[u][e] = av[ru][u].v[e] * xrv[ru] + colacc[u][e];
             }
       } else {
+        // Edge and diagonal tiles: local 32-bit indices; d = (first column) - (first row), so
+        // element (li, lj) lies on the diagonal when d + lj == li.
+        const int64_t d64 = c0 - rb;
+        const int d = (int)(d64 > (1 << 24) ? (1 << 24) : d64 < -(1 << 24) ? -(1 << 24) : d64);
+        const int nc = (int)(c1 - c0);
+        const T* at = a_rb + c0;
 #pragma unroll
         for (int ru = 0; ru < RU; ++ru) {
-          const int64_t i = rowi[ru];
-          if (i >= r_end) continue;
+          const int li = lrow0 + ru * kWarps * G;
+          if (li >= nr) continue;
 #pragma unroll
           for (int u = 0; u < CU; ++u) {
-            const int64_t cv = c0 + (u * LPR + q) * V;
-            if (cv >= p.cols) continue;
-            if (K::TRI == TRI_UPPER && cv + V - 1 < i) continue;  // pack wholly outside
-            if (K::TRI == TRI_LOWER && cv > i) continue;
+            const int lc = (u * LPR + q) * V;
+            if (lc >= nc) continue;
+            if (K::TRI == TRI_UPPER && d + lc + V - 1 < li) continue;  // pack wholly outside
+            if (K::TRI == TRI_LOWER && d + lc > li) continue;
+            const T* ap = at + ru * rstride + u * (LPR * V);
             P av;
-            if (V > 1 && cv + V <= p.cols) {
-              av = ld_nc<T, V>(p.a + i * p.lda + cv);
+            if (V > 1 && lc + V <= nc) {
+              av = ld_nc<T, V>(ap);
             } else {
 #pragma unroll
-              for (int e = 0; e < V; ++e) av.v[e] = (cv + e < p.cols) ? __ldg(p.a + i * p.lda + cv + e) : T(0);
+              for (int e = 0; e < V; ++e) av.v[e] = (lc + e < nc) ? __ldg(ap + e) : T(0);
             }
 #pragma unroll
             for (int e = 0; e < V; ++e) {
-              const int64_t j = cv + e;
-              if (j >= p.cols) continue;
-              if (K::TRI == TRI_UPPER && j < i) continue;
-              if (K::TRI == TRI_LOWER && j > i) continue;
-              const bool dg = (K::TRI != TRI_FULL) && (j == i);
+              const int lj = lc + e;
+              if (lj >= nc) continue;
+              if (K::TRI == TRI_UPPER && d + lj < li) continue;
+              if (K::TRI == TRI_LOWER && d + lj > li) continue;
+              const bool dg = (K::TRI != TRI_FULL) && (d + lj == li);
               const T v = (K::UNIT && dg) ? T(1) : av.v[e];
               if (K::ROWOUT) rowacc[ru] = v * xcv[u][e] + rowacc[ru];
               if (K::COLOUT && !(K::SYM && dg)) colacc[u][e] = v * xrv[ru] + colacc[u][e];
