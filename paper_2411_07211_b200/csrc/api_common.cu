@@ -7,7 +7,7 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobL1BlocksPerSm   */ 8,
     /* kKnobGemvNTileBytes  */ 64 * 1024,
     /* kKnobGemvTRows       */ 256,
-    /* kKnobTriRows         */ 256,
+    /* kKnobTriRows         */ 512,
     /* kKnobGerRows         */ 2,
     /* kKnobUsePdl          */ 1,
     /* kKnobTrsvDebugSkip   */ -1,

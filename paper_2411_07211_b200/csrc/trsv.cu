@@ -1,12 +1,12 @@
 // trsv: solve op(A) x = b in place (Section 6.2.2; same option space as trmv).
 //
 // Blocked substitution with a dependency-ordered diagonal-block solve.  The unknowns are cut
-// into blocks of 128; thread blocks draw a ticket k = 0, 1, ... (the solve order: top-down for
+// into blocks of 128 (float) or 64 (double); thread blocks draw a ticket k = 0, 1, ... (the solve order: top-down for
 // an effectively lower-triangular op(A), bottom-up for an upper one).  Block k
-//   1. stages its 128x128 diagonal block in shared memory and inverts it there, in place, by
+//   1. stages its diagonal block in shared memory and inverts it there, in place, by
 //      recursive doubling (none of this depends on the solve),
 //   2. streams the off-diagonal part of its block row (or block column when op(A)'s rows are
-//      strided in memory) as 128x64 tiles in solve order; 16 compute warps keep the next
+//      strided in memory) as tiles of 64 source unknowns in solve order; 16 compute warps keep the next
 //      tile's matrix data in flight in registers and tiles further ahead are pulled into L2,
 //      all BEFORE the x values they multiply exist,
 //   3. receives those x values through a side buffer in the workspace in which every value is
@@ -17,29 +17,27 @@
 //      (named barriers), so polling latency never stalls the streaming warps, and only one warp
 //      per block loads the hot words -- a herd of pollers would swamp the L2 slice that
 //      holds them,
-//   4. forms r = b - sum, multiplies by the inverted diagonal block, publishes its 128 values
+//   4. forms r = b - sum, multiplies by the inverted diagonal block, publishes its values
 //      and writes them to the caller's x.
-// The chain of n/128 dependent steps makes the routine latency-bound: each step costs one L2
-// store->load hand-over plus a 128x128 matvec.  Tickets are drawn in launch order, so a block
+// The chain of dependent block solves makes the routine latency-bound: each step costs one L2
+// store->load hand-over plus a block-sized matvec.  Tickets are drawn in launch order, so a block
 // only ever waits for blocks that are already running: no co-residency assumption, no
 // deadlock.  If the polls exceed the iteration limit the block records B2_STATUS_TIMEOUT in
 // *device_status and leaves without publishing (its dependants then time out too).
 //
 // Accuracy note: the diagonal blocks are applied through their explicit inverses (computed in
 // the working precision).  For diagonal blocks of moderate condition number this is as
-// accurate as substitution; it is the usual trade for removing 128 dependent steps per block.
+// accurate as substitution; it is the usual trade for removing the dependent steps inside a block.
 #include <atomic>
 
 #include "common.cuh"
 
 namespace b2 {
 
-constexpr int kNB = 128;              // unknowns per thread block
 constexpr int kSB = 64;               // unknowns per source tile
 constexpr int kCW = 16;               // compute warps
 constexpr int kCT = kCW * 32;         // compute threads
 constexpr int kTT = kCT + 32;         // + one polling warp
-constexpr int kWS = kNB + 8;          // row stride of the diagonal-block array (16-byte row starts, conflict-free packs)
 constexpr int kXB = 4;                // x buffers between the polling warp and the compute warps
 constexpr int kBarFull = 1;           // named barriers kBarFull + b, kBarEmpty + b
 constexpr int kBarEmpty = 1 + kXB;
@@ -67,7 +65,7 @@ struct TrsvArgs {
   int64_t incx;
   unsigned long long* xbuf;  // published solution: 1 (float) or 2 (double) tagged words per unknown
   unsigned* ticket;
-  int nb;   // 128-blocks
+  int nb;   // blocks of trsv_block<T>() unknowns
   int nsb;  // 64-blocks (source tiles)
   unsigned tag;
   unsigned long long wait_limit;
@@ -131,11 +129,15 @@ __device__ __forceinline__ double decode(const unsigned long long* w, double) {
 }
 
 // COLTYPE: op(A)'s rows are columns of the stored row-major view.  BACKWARD: solve bottom-up.
-template <typename T, int V, bool COLTYPE, bool BACKWARD, bool UNIT>
+// NB = unknowns per thread block: 128 for float, 64 for double (the diagonal-block work grows with
+// NB^2 per unknown and double-precision multiply-adds are scarce on this part).
+template <typename T, int NB, int V, bool COLTYPE, bool BACKWARD, bool UNIT>
 __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
-  // A tile is 128 own unknowns x 64 source unknowns; in memory it is 128 rows x 64 columns
-  // (rows of op(A) contiguous) or 64 rows x 128 columns (COLTYPE).
-  constexpr int TROWS = COLTYPE ? kSB : kNB, TCOLS = COLTYPE ? kNB : kSB;
+  // A tile is NB own unknowns x 64 source unknowns; in memory it is NB rows x 64 columns
+  // (rows of op(A) contiguous) or 64 rows x NB columns (COLTYPE).
+  constexpr int WS = NB + 8;        // row stride of W (16-byte row starts, conflict-free packs)
+  constexpr int TPB = NB / kSB;     // source tiles a solved block publishes at once
+  constexpr int TROWS = COLTYPE ? kSB : NB, TCOLS = COLTYPE ? NB : kSB;
   constexpr int LPR = (TCOLS / V) >= 32 ? 32 : TCOLS / V;
   constexpr int CU = TCOLS / (LPR * V);
   constexpr int G = 32 / LPR;
@@ -145,11 +147,11 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
   using P = Pack<T, V>;
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  T* W = reinterpret_cast<T*>(smem_raw);  // diagonal block in solve order, W[s*kWS + t], then its inverse
-  T* racc = W + kNB * kWS;                // r = b - (sum over solved blocks), per unknown (solve order)
-  T* bvec = racc + kNB;                   // right-hand side b (solve order)
-  T* xsm = bvec + kNB;                    // [kXB][kSB] x values handed over by the polling warp
-  T* colsm = xsm + kXB * kSB;             // [kCW][kNB], COLTYPE only
+  T* W = reinterpret_cast<T*>(smem_raw);  // diagonal block in solve order, W[s*WS + t], then its inverse
+  T* racc = W + NB * WS;                // r = b - (sum over solved blocks), per unknown (solve order)
+  T* bvec = racc + NB;                   // right-hand side b (solve order)
+  T* xsm = bvec + NB;                    // [kXB][kSB] x values handed over by the polling warp
+  T* colsm = xsm + kXB * kSB;             // [kCW][NB], COLTYPE only
   __shared__ unsigned s_ticket;
   __shared__ int s_abort;
 
@@ -167,11 +169,11 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
     return;
   }
   const int I = BACKWARD ? p.nb - 1 - k : k;  // block index in memory
-  const int64_t r0 = (int64_t)I * kNB;
-  const int nbI = (int)min((int64_t)kNB, p.n - r0);
+  const int64_t r0 = (int64_t)I * NB;
+  const int nbI = (int)min((int64_t)NB, p.n - r0);
   auto solve_idx = [&](int i) { return BACKWARD ? nbI - 1 - i : i; };
   // source tiles (64 unknowns each) in solve order: s -> global 64-block index
-  const int nsrc = BACKWARD ? max(0, p.nsb - 2 * I - 2) : 2 * I;
+  const int nsrc = BACKWARD ? max(0, p.nsb - TPB * I - TPB) : TPB * I;
   auto src_block = [&](int s) { return BACKWARD ? p.nsb - 1 - s : s; };
 
   int lr[RU];
@@ -205,7 +207,7 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
   auto prefetch_tile = [&](int s) {
     if (s >= nsrc) return;
     const int64_t c0 = (int64_t)src_block(s) * kSB;
-    if (p.n - c0 < kSB || nbI < kNB) return;  // ragged tiles are not worth it
+    if (p.n - c0 < kSB || nbI < NB) return;  // ragged tiles are not worth it
     const int64_t rbase = COLTYPE ? c0 : r0, cbase = COLTYPE ? r0 : c0;
     constexpr int LINES = TCOLS * (int)sizeof(T) / 128;
     for (int i = tid; i < TROWS * LINES; i += kCT) {
@@ -222,36 +224,36 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
   }
 
   // 1a. diagonal block -> W (zero elsewhere, identity on unused / unit diagonal); b -> bvec
-  for (int idx = tid; idx < kNB * kWS; idx += kTT) W[idx] = T(0);
-  if (tid < kNB) {
+  for (int idx = tid; idx < NB * WS; idx += kTT) W[idx] = T(0);
+  if (tid < NB) {
     bvec[tid] = tid < nbI ? p.x[(r0 + solve_idx(tid)) * p.incx] : T(0);
     racc[tid] = bvec[tid];  // r = b when nothing precedes; entries past a ragged block stay zero
   }
   __syncthreads();
-  for (int base = 0; base < kNB * kNB; base += 8 * kTT) {  // 8 independent loads in flight per thread
+  for (int base = 0; base < NB * NB; base += 8 * kTT) {  // 8 independent loads in flight per thread
     T v[8];
     bool use[8];
 #pragma unroll
     for (int m = 0; m < 8; ++m) {
       const int idx = base + m * kTT + tid;
-      const int pr = idx / kNB, pc = idx % kNB;  // position inside the stored block
-      use[m] = idx < kNB * kNB && pr < nbI && pc < nbI && (CANON_LOWER ? (pc <= pr) : (pc >= pr)) &&
+      const int pr = idx / NB, pc = idx % NB;  // position inside the stored block
+      use[m] = idx < NB * NB && pr < nbI && pc < nbI && (CANON_LOWER ? (pc <= pr) : (pc >= pr)) &&
                !(UNIT && pr == pc);
       v[m] = use[m] ? __ldg(p.a + (r0 + pr) * p.lda + r0 + pc) : T(0);
     }
 #pragma unroll
     for (int m = 0; m < 8; ++m) {
       const int idx = base + m * kTT + tid;
-      const int pr = idx / kNB, pc = idx % kNB;
+      const int pr = idx / NB, pc = idx % NB;
       if (use[m]) {
         const int sr = solve_idx(pr), sc = solve_idx(pc);
-        if (COLTYPE) W[sc * kWS + sr] = v[m];
-        else W[sr * kWS + sc] = v[m];
+        if (COLTYPE) W[sc * WS + sr] = v[m];
+        else W[sr * WS + sc] = v[m];
       }
     }
   }
-  for (int s = tid; s < kNB; s += kTT)
-    if (UNIT || s >= nbI) W[s * kWS + s] = T(1);
+  for (int s = tid; s < NB; s += kTT)
+    if (UNIT || s >= nbI) W[s * WS + s] = T(1);
   __syncthreads();
 
   // 1b. in-place inverse by recursive doubling.  4x4 diagonal blocks: one column per thread,
@@ -261,12 +263,12 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
   {
     T col[4];
     const int c = tid, d0 = (c / 4) * 4, lc = c % 4;
-    if (tid < kNB) {
+    if (tid < NB) {
       T e[4][4];
 #pragma unroll
       for (int ls = 0; ls < 4; ++ls)
 #pragma unroll
-        for (int lt = 0; lt <= ls; ++lt) e[ls][lt] = W[(d0 + ls) * kWS + d0 + lt];
+        for (int lt = 0; lt <= ls; ++lt) e[ls][lt] = W[(d0 + ls) * WS + d0 + lt];
 #pragma unroll
       for (int ls = 0; ls < 4; ++ls) {
         T acc = (ls == lc) ? T(1) : T(0);
@@ -276,15 +278,15 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
       }
     }
     __syncthreads();
-    if (tid < kNB) {
+    if (tid < NB) {
 #pragma unroll
-      for (int ls = 0; ls < 4; ++ls) W[(d0 + ls) * kWS + c] = col[ls];  // zero above the diagonal
+      for (int ls = 0; ls < 4; ++ls) W[(d0 + ls) * WS + c] = col[ls];  // zero above the diagonal
     }
     __syncthreads();
   }
 #pragma unroll 1
-  for (int h = 4; h < kNB; h *= 2) {  // 4x4 register tiles: 8 shared-memory loads per 16 multiply-adds
-    const int tpr = h / 4, per_pair = tpr * tpr, total = (kNB / (2 * h)) * per_pair;
+  for (int h = 4; h < NB; h *= 2) {  // 4x4 register tiles: 8 shared-memory loads per 16 multiply-adds
+    const int tpr = h / 4, per_pair = tpr * tpr, total = (NB / (2 * h)) * per_pair;
     for (int e = tid; e < total; e += kTT) {  // Tm = C * A^-1  (A^-1 is zero above its diagonal)
       const int pr = e / per_pair, i0 = ((e % per_pair) / tpr) * 4, j0 = (e % tpr) * 4;
       const int top = pr * 2 * h, bot = top + h;
@@ -297,9 +299,9 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
       for (int l = j0; l < h; ++l) {
         T cv[4], av[4];
 #pragma unroll
-        for (int ii = 0; ii < 4; ++ii) cv[ii] = W[(bot + i0 + ii) * kWS + top + l];
+        for (int ii = 0; ii < 4; ++ii) cv[ii] = W[(bot + i0 + ii) * WS + top + l];
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) av[jj] = W[(top + l) * kWS + top + j0 + jj];
+        for (int jj = 0; jj < 4; ++jj) av[jj] = W[(top + l) * WS + top + j0 + jj];
 #pragma unroll
         for (int ii = 0; ii < 4; ++ii)
 #pragma unroll
@@ -308,7 +310,7 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
 #pragma unroll
       for (int ii = 0; ii < 4; ++ii)
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) W[(top + j0 + jj) * kWS + bot + i0 + ii] = acc[ii][jj];
+        for (int jj = 0; jj < 4; ++jj) W[(top + j0 + jj) * WS + bot + i0 + ii] = acc[ii][jj];
     }
     __syncthreads();
     for (int e = tid; e < total; e += kTT) {  // X = -B^-1 * Tm, written over C (B^-1 zero above its diagonal)
@@ -323,9 +325,9 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
       for (int l = 0; l < i0 + 4; ++l) {
         T bv[4], tv[4];
 #pragma unroll
-        for (int ii = 0; ii < 4; ++ii) bv[ii] = W[(bot + i0 + ii) * kWS + bot + l];
+        for (int ii = 0; ii < 4; ++ii) bv[ii] = W[(bot + i0 + ii) * WS + bot + l];
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) tv[jj] = W[(top + j0 + jj) * kWS + bot + l];
+        for (int jj = 0; jj < 4; ++jj) tv[jj] = W[(top + j0 + jj) * WS + bot + l];
 #pragma unroll
         for (int ii = 0; ii < 4; ++ii)
 #pragma unroll
@@ -334,26 +336,26 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
 #pragma unroll
       for (int ii = 0; ii < 4; ++ii)
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) W[(bot + i0 + ii) * kWS + top + j0 + jj] = -acc[ii][jj];
+        for (int jj = 0; jj < 4; ++jj) W[(bot + i0 + ii) * WS + top + j0 + jj] = -acc[ii][jj];
     }
     __syncthreads();
-    for (int e = tid; e < (kNB / (2 * h)) * h * h; e += kTT) {  // scrub the parked intermediates
+    for (int e = tid; e < (NB / (2 * h)) * h * h; e += kTT) {  // scrub the parked intermediates
       const int pr = e / (h * h), i = (e % (h * h)) / h, j = e % h;
-      W[(pr * 2 * h + j) * kWS + pr * 2 * h + h + i] = T(0);
+      W[(pr * 2 * h + j) * WS + pr * 2 * h + h + i] = T(0);
     }
     __syncthreads();
   }
-  // The finished inverse: float blocks keep their share in registers (the 128x128 matvec is then
+  // The finished inverse: float blocks keep their share in registers (the matvec is then
   // free of shared-memory traffic), double blocks read it from shared memory in 16-byte packs.
   constexpr int VL = 16 / (int)sizeof(T);          // elements per pack
-  constexpr int TPU = kCT / kNB;                   // threads per unknown (4)
-  constexpr int NPK = kNB / (TPU * VL);            // packs per thread
+  constexpr int TPU = kCT / NB;                   // threads per unknown
+  constexpr int NPK = NB / (TPU * VL);            // packs per thread
   constexpr bool WREG = sizeof(T) == 4;
   Pack<T, VL> wreg[WREG ? NPK : 1];
   if (WREG && !poller) {
     const int ms = tid / TPU, part = tid % TPU;
 #pragma unroll
-    for (int m = 0; m < NPK; ++m) wreg[m] = *reinterpret_cast<const Pack<T, VL>*>(&W[ms * kWS + VL * (part + TPU * m)]);
+    for (int m = 0; m < NPK; ++m) wreg[m] = *reinterpret_cast<const Pack<T, VL>*>(&W[ms * WS + VL * (part + TPU * m)]);
   }
 
   // 2./3. off-diagonal tiles in solve order
@@ -372,22 +374,22 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
     poll.abort_flag = &s_abort;
     poll.device_status = p.device_status;
     poll.tag = p.tag;
-    // A solved block publishes 128 unknowns = two source tiles at once, so the tiles are polled
-    // in pairs: one round trip through L2 serves both.
-    constexpr int EPL = 2 * kSB / 32;  // unknowns per lane and pair
-    for (int s = 0; s < nsrc; s += 2) {
-      const int b0 = s % kXB, b1 = (s + 1) % kXB;
-      if (s >= kXB) bar_sync(kBarEmpty + b0, kTT);  // the compute warps are done with these buffers
-      if (s + 1 < nsrc && s + 1 >= kXB) bar_sync(kBarEmpty + b1, kTT);
+    // A solved block publishes NB unknowns = TPB source tiles at once, so the tiles are polled TPB
+    // at a time: one round trip through L2 serves them all.
+    constexpr int EPL = TPB * kSB / 32;  // unknowns per lane and poll
+    for (int s = 0; s < nsrc; s += TPB) {
+#pragma unroll
+      for (int t = 0; t < TPB; ++t)  // the compute warps are done with these buffers
+        if (s + t < nsrc && s + t >= kXB) bar_sync(kBarEmpty + (s + t) % kXB, kTT);
       // blocks further from the front sleep between polls so that only the next in line spins
-      const int last = min(s + 1, nsrc - 1);
-      const int dist = k - (BACKWARD ? p.nb - 1 - src_block(last) / 2 : src_block(last) / 2);
+      const int last = min(s + TPB - 1, nsrc - 1);
+      const int dist = k - (BACKWARD ? p.nb - 1 - src_block(last) / TPB : src_block(last) / TPB);
       poll.backoff_ns = dist > 1 ? (unsigned)min(dist - 1, 64) * 500u : 0u;
       unsigned long long w[EPL * WPE];
       const unsigned long long* wp[EPL * WPE];
 #pragma unroll
       for (int j = 0; j < EPL; ++j) {
-        const int el = lane * EPL + j, t = el / kSB, lc = el % kSB;  // tile of the pair, position in it
+        const int el = lane * EPL + j, t = el / kSB, lc = el % kSB;  // tile of the group, position in it
         const int64_t u = (int64_t)src_block(min(s + t, nsrc - 1)) * kSB + lc;
         const bool valid = s + t < nsrc && u < p.n;
 #pragma unroll
@@ -397,11 +399,12 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
 #pragma unroll
       for (int j = 0; j < EPL; ++j) {
         const int el = lane * EPL + j, t = el / kSB, lc = el % kSB;
-        xsm[(t ? b1 : b0) * kSB + lc] = wp[j * WPE] ? decode(&w[j * WPE], T(0)) : T(0);
+        xsm[((s + t) % kXB) * kSB + lc] = wp[j * WPE] ? decode(&w[j * WPE], T(0)) : T(0);
       }
       __threadfence_block();
-      bar_arrive(kBarFull + b0, kTT);
-      if (s + 1 < nsrc) bar_arrive(kBarFull + b1, kTT);
+#pragma unroll
+      for (int t = 0; t < TPB; ++t)
+        if (s + t < nsrc) bar_arrive(kBarFull + (s + t) % kXB, kTT);
     }
   } else {
 #pragma unroll 1
@@ -450,7 +453,7 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
 #pragma unroll
         for (int e = 0; e < V; ++e) {
           const T s = cross_group_sum<LPR>(colacc[u][e]);
-          if (g == 0) colsm[warp * kNB + (u * LPR + q) * V + e] = s;
+          if (g == 0) colsm[warp * NB + (u * LPR + q) * V + e] = s;
         }
     } else {
       constexpr int LPV = LPR / RU;  // lanes left per row after the reduction
@@ -464,7 +467,7 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
     if (tid < nbI) {
       T s = colsm[tid];
 #pragma unroll
-      for (int w = 1; w < kCW; ++w) s += colsm[w * kNB + tid];
+      for (int w = 1; w < kCW; ++w) s += colsm[w * NB + tid];
       racc[solve_idx(tid)] = bvec[solve_idx(tid)] - s;
     }
     __syncthreads();
@@ -485,7 +488,7 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
 #pragma unroll
         for (int e = 0; e < VL; ++e) accv[e] = wreg[m].v[e] * rv.v[e] + accv[e];
       } else if (t0 <= s) {  // W is zero above the diagonal
-        const Pack<T, VL> wv = *reinterpret_cast<const Pack<T, VL>*>(&W[s * kWS + t0]);
+        const Pack<T, VL> wv = *reinterpret_cast<const Pack<T, VL>*>(&W[s * WS + t0]);
         const Pack<T, VL> rv = *reinterpret_cast<const Pack<T, VL>*>(&racc[t0]);
 #pragma unroll
         for (int e = 0; e < VL; ++e) accv[e] = wv.v[e] * rv.v[e] + accv[e];
@@ -505,15 +508,20 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
   if (k == p.nb - 1 && tid == 0) *p.ticket = 0u;  // all tickets are drawn: leave the control block clean
 }
 
+template <typename T>
+constexpr int trsv_block() {
+  return sizeof(T) == 4 ? 128 : 64;
+}
 template <typename T, bool COLTYPE>
 constexpr size_t trsv_smem_bytes() {
-  return sizeof(T) * (kNB * kWS + 2 * kNB + kXB * kSB + (COLTYPE ? kCW : 0) * kNB);
+  constexpr int NB = trsv_block<T>();
+  return sizeof(T) * (NB * (NB + 8) + 2 * NB + kXB * kSB + (COLTYPE ? kCW : 0) * NB);
 }
 
 template <typename T, int V, bool COLTYPE, bool BACKWARD, bool UNIT>
 static int trsv_launch_one(const Launch& l, const TrsvArgs<T>& args) {
   constexpr size_t smem = trsv_smem_bytes<T, COLTYPE>();
-  auto kern = trsv_kernel<T, V, COLTYPE, BACKWARD, UNIT>;
+  auto kern = trsv_kernel<T, trsv_block<T>(), V, COLTYPE, BACKWARD, UNIT>;
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -559,7 +567,8 @@ static int trsv_impl(const b2_ctx* ctx, int order, int uplo, int trans, int diag
   Launch l;
   if (int st = make_launch(ctx, &l)) return st;
   if (n == 0) return B2_STATUS_OK;
-  if ((n + kNB - 1) / kNB > 0x3fffffff) return B2_STATUS_NOT_IMPLEMENTED;
+  constexpr int NB = trsv_block<T>();
+  if ((n + NB - 1) / NB > 0x3fffffff) return B2_STATUS_NOT_IMPLEMENTED;
   const size_t xbuf_bytes = (size_t)n * 8 * (sizeof(T) / 4);
   if (l.scratch_bytes < xbuf_bytes) return B2_STATUS_WORKSPACE_TOO_SMALL;
   TrsvArgs<T> args = {};
@@ -570,14 +579,14 @@ static int trsv_impl(const b2_ctx* ctx, int order, int uplo, int trans, int diag
   args.incx = incx;
   args.xbuf = reinterpret_cast<unsigned long long*>(l.scratch);
   args.ticket = l.ctl + kCtlTrsvTicket;
-  args.nb = (int)((n + kNB - 1) / kNB);
+  args.nb = (int)((n + NB - 1) / NB);
   args.nsb = (int)((n + kSB - 1) / kSB);
   args.tag = next_tag();
   args.wait_limit = l.wait_limit;
   args.device_status = l.device_status;
   args.debug_skip = (int)knob(kKnobTrsvDebugSkip);
   {  // keep the prefetched-but-unused tiles of all blocks within a fraction of L2
-    const int64_t tile_bytes = (int64_t)kNB * kSB * sizeof(T);
+    const int64_t tile_bytes = (int64_t)NB * kSB * sizeof(T);
     int64_t d = knob(kKnobTrsvPrefetchBytes) / (tile_bytes * args.nb);
     args.pf_dist = (int)(d < 0 ? 0 : d > 64 ? 64 : d);
   }
