@@ -28,6 +28,11 @@ sys.path.insert(0, ROOT)
 MIB = 1 << 20
 ROW, COL, NOTR, TR, UP, LO, NONU, UNIT = 101, 102, 111, 112, 121, 122, 131, 132
 FALLBACK_PEAK_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of each kernel template at the bench
+# sizes, from the ncu captures summarised in profiles/kernels_config5_ncu_full.md (same kernels).
+# Set an entry to None when its kernel changes and the counters have not been retaken.
+NCU_DRAM_BYTES_PER_LAUNCH = {"trsv": 271.4e6, "l2_tile": 271.3e6, "l1_reduce": 272.3e6, "l1_map": 351.8e6,
+                             "ger": 479.3e6}
 
 
 # --------------------------------------------------------------------------- variant table
@@ -474,12 +479,7 @@ def main():
                      "share_of_time": v["ms"] / sum(x["ms"] for x in fam.values()), "variants": v["launches"]}
                  for k, v in fam.items()}
     dom = max(fam, key=lambda k: fam[k]["ms"])
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    traffic = None
-    try:
-        traffic = json.load(open(traffic_path)).get(dom)
-    except Exception:
-        pass
+    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(dom)
     roofline = {"bound": "hbm", "kernel": dom, "achieved": by_kernel[dom]["achieved"], "peak": peak, "unit": "GB/s",
                 "frac": by_kernel[dom]["frac"], "traffic": traffic, "peak_source": peak_src,
                 "by_kernel": by_kernel}
