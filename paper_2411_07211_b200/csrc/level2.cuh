@@ -54,7 +54,7 @@ struct L2Args {
   int64_t rows_per_cta;
   int ctiles_per_cta, nct, nrs, ncs;
   int direct;  // 1: blocks write alpha*acc + beta*y straight to y
-  int xc_vec;  // 1: xc has unit stride and 16-byte alignment, so it can be read in packs
+  int xc_vec;  // xc is 16-byte aligned with increment 1 (value 1) or 2 (value 2): read it in packs
   T alpha, beta;
   T* y;
   int64_t incy;
@@ -131,12 +131,22 @@ __global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p)
       if (!region_active<K::TRI>(rb, rb_end, c0, c1)) continue;
       if (K::ROWOUT && xcv_ct != ct) {
         xcv_ct = ct;
-        if (V > 1 && p.xc_vec && c0 + TC <= p.cols) {
+        if (V > 1 && p.xc_vec == 1 && c0 + TC <= p.cols) {
 #pragma unroll
           for (int u = 0; u < CU; ++u) {
             const P xv = ld_ro<T, V>(p.xc + c0 + (u * LPR + q) * V);
 #pragma unroll
             for (int e = 0; e < V; ++e) xcv[u][e] = xv.v[e];
+          }
+        } else if (V > 1 && p.xc_vec == 2 && c0 + TC < p.cols) {
+          // increment 2: the V values sit in two consecutive packs (even positions); the odd
+          // position after the last value exists because the tile is not the vector's last
+#pragma unroll
+          for (int u = 0; u < CU; ++u) {
+            const T* xp = p.xc + 2 * (c0 + (u * LPR + q) * V);
+            const P x0 = ld_ro<T, V>(xp), x1 = ld_ro<T, V>(xp + V);
+#pragma unroll
+            for (int e = 0; e < V; ++e) xcv[u][e] = (2 * e < V) ? x0.v[(2 * e) % V] : x1.v[(2 * e) % V];
           }
         } else {
 #pragma unroll
@@ -329,7 +339,7 @@ static int l2_launch_shape(const Launch& l, L2Args<T> args, int64_t rows_per_cta
   constexpr int TC = S::template tc<V>();
   constexpr int RB = S::RB;
   args.nct = (int)((args.cols + TC - 1) / TC);
-  args.xc_vec = (K::ROWOUT && V > 1 && args.incxc == 1 && aligned_to(args.xc, 16)) ? 1 : 0;
+  args.xc_vec = (K::ROWOUT && V > 1 && aligned_to(args.xc, 16)) ? (args.incxc == 1 ? 1 : args.incxc == 2 ? 2 : 0) : 0;
   if (K::COLOUT) ctiles_per_cta = 1;
   if (ctiles_per_cta < 1) ctiles_per_cta = 1;
   if (ctiles_per_cta > args.nct) ctiles_per_cta = args.nct;
