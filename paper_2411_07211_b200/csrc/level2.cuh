@@ -31,9 +31,12 @@ struct Kind {
 
 // LPR lanes cover one row segment, so a warp covers G = 32/LPR rows per step; each lane owns
 // CU packs of V columns; RU row steps are in flight per warp.
-template <int LPR_, int CU_, int RU_>
+// NCT: column tiles a block of a COLOUT kind walks per row step (their column sums stay in
+// registers side by side, the row sums run across all of them).
+template <int LPR_, int CU_, int RU_, int NCT_ = 1>
 struct Shape {
-  static constexpr int LPR = LPR_, CU = CU_, RU = RU_, G = 32 / LPR_;
+  static constexpr int LPR = LPR_, CU = CU_, RU = RU_, G = 32 / LPR_, NCT = NCT_;
+  static constexpr int MINB = NCT_ == 1 ? 4 : 3;  // resident blocks per SM the register budget aims at
   static constexpr int RB = kWarps * G * RU_;  // rows per block step
   template <int V>
   static constexpr int tc() {
@@ -77,9 +80,10 @@ __device__ __forceinline__ bool region_strictly_inside(int64_t r0, int64_t r1, i
 }
 
 template <typename T, int V, class K, class S>
-__global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p) {
+__global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args<T> p) {
   constexpr int LPR = S::LPR, CU = S::CU, RU = S::RU, G = S::G, RB = S::RB;
   constexpr int TC = LPR * V * CU;
+  constexpr int NCT = K::COLOUT ? S::NCT : 1;
   using P = Pack<T, V>;
   grid_dep_launch();  // lets a dependent finalize launch be scheduled early (it waits for us)
 
@@ -94,13 +98,17 @@ __global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p)
   const int64_t c_lo = (int64_t)ct_begin * TC, c_hi = min(p.cols, (int64_t)ct_end * TC);
   if (!region_active<K::TRI>(r_begin, r_end, c_lo, c_hi)) return;
 
-  T colacc[CU][V];
-  T xcv[CU][V];
+  T colacc[NCT][CU][V];
+  T xcv[NCT][CU][V];
+  int xcv_ct[NCT];  // column tile whose x values are in xcv[c]
 #pragma unroll
-  for (int u = 0; u < CU; ++u)
+  for (int c = 0; c < NCT; ++c) {
+    xcv_ct[c] = -1;
 #pragma unroll
-    for (int e = 0; e < V; ++e) colacc[u][e] = T(0), xcv[u][e] = T(0);
-  int xcv_ct = -1;  // column tile whose x values are in xcv
+    for (int u = 0; u < CU; ++u)
+#pragma unroll
+      for (int e = 0; e < V; ++e) colacc[c][u][e] = T(0), xcv[c][u][e] = T(0);
+  }
 
   // Address arithmetic is hoisted: inside a tile everything is a 32-bit local index or a
   // pointer bumped by a precomputed stride.
@@ -126,17 +134,23 @@ __global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p)
       for (int ru = 0; ru < RU; ++ru)
         if (lrow0 + ru * kWarps * G < nr) xrv[ru] = __ldg(xp + ru * xstride);
     }
-    for (int ct = ct_begin; ct < ct_end; ++ct) {
+    // COLOUT kinds: slot c holds column tile ct_begin + c; ROWOUT-only kinds: one slot, any
+    // number of column tiles.
+#pragma unroll
+    for (int c = 0; c < NCT; ++c) {
+    const int ct_lo = K::COLOUT ? ct_begin + c : ct_begin;
+    const int ct_hi = K::COLOUT ? min(ct_lo + 1, ct_end) : ct_end;
+    for (int ct = ct_lo; ct < ct_hi; ++ct) {
       const int64_t c0 = (int64_t)ct * TC, c1 = min(p.cols, c0 + TC);
       if (!region_active<K::TRI>(rb, rb_end, c0, c1)) continue;
-      if (K::ROWOUT && xcv_ct != ct) {
-        xcv_ct = ct;
+      if (K::ROWOUT && xcv_ct[c] != ct) {
+        xcv_ct[c] = ct;
         if (V > 1 && p.xc_vec == 1 && c0 + TC <= p.cols) {
 #pragma unroll
           for (int u = 0; u < CU; ++u) {
             const P xv = ld_ro<T, V>(p.xc + c0 + (u * LPR + q) * V);
 #pragma unroll
-            for (int e = 0; e < V; ++e) xcv[u][e] = xv.v[e];
+            for (int e = 0; e < V; ++e) xcv[c][u][e] = xv.v[e];
           }
         } else if (V > 1 && p.xc_vec == 2 && c0 + TC < p.cols) {
           // increment 2: the V values sit in two consecutive packs (even positions); the odd
@@ -146,7 +160,7 @@ __global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p)
             const T* xp = p.xc + 2 * (c0 + (u * LPR + q) * V);
             const P x0 = ld_ro<T, V>(xp), x1 = ld_ro<T, V>(xp + V);
 #pragma unroll
-            for (int e = 0; e < V; ++e) xcv[u][e] = (2 * e < V) ? x0.v[(2 * e) % V] : x1.v[(2 * e) % V];
+            for (int e = 0; e < V; ++e) xcv[c][u][e] = (2 * e < V) ? x0.v[(2 * e) % V] : x1.v[(2 * e) % V];
           }
         } else {
 #pragma unroll
@@ -154,7 +168,7 @@ __global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p)
 #pragma unroll
             for (int e = 0; e < V; ++e) {
               const int64_t j = c0 + (u * LPR + q) * V + e;
-              xcv[u][e] = j < p.cols ? __ldg(p.xc + j * p.incxc) : T(0);
+              xcv[c][u][e] = j < p.cols ? __ldg(p.xc + j * p.incxc) : T(0);
             }
         }
       }
@@ -173,8 +187,8 @@ __global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p)
           for (int u = 0; u < CU; ++u)
 #pragma unroll
             for (int e = 0; e < V; ++e) {
-              if (K::ROWOUT) rowacc[ru] = av[ru][u].v[e] * xcv[u][e] + rowacc[ru];
-              if (K::COLOUT) colacc[u][e] = av[ru][u].v[e] * xrv[ru] + colacc[u][e];
+              if (K::ROWOUT) rowacc[ru] = av[ru][u].v[e] * xcv[c][u][e] + rowacc[ru];
+              if (K::COLOUT) colacc[c][u][e] = av[ru][u].v[e] * xrv[ru] + colacc[c][u][e];
             }
       } else {
         // Edge and diagonal tiles: local 32-bit indices; d = (first column) - (first row), so
@@ -209,13 +223,14 @@ __global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p)
               if (K::TRI == TRI_LOWER && d + lj > li) continue;
               const bool dg = (K::TRI != TRI_FULL) && (d + lj == li);
               const T v = (K::UNIT && dg) ? T(1) : av.v[e];
-              if (K::ROWOUT) rowacc[ru] = v * xcv[u][e] + rowacc[ru];
-              if (K::COLOUT && !(K::SYM && dg)) colacc[u][e] = v * xrv[ru] + colacc[u][e];
+              if (K::ROWOUT) rowacc[ru] = v * xcv[c][u][e] + rowacc[ru];
+              if (K::COLOUT && !(K::SYM && dg)) colacc[c][u][e] = v * xrv[ru] + colacc[c][u][e];
             }
           }
         }
       }
     }
+    }  // slot c
     if (K::ROWOUT) {  // all RU row sums in one transposing butterfly
       constexpr int LPV = LPR / RU;  // lanes left per row after the reduction
       const T s = multi_group_sum<LPR, RU>(rowacc, lane);
@@ -231,17 +246,19 @@ __global__ void __launch_bounds__(kThreads, 4) l2_tile_kernel(const L2Args<T> p)
     }
   }
 
-  if constexpr (K::COLOUT) {  // one column tile per block for these kinds
-    __shared__ T sm[kWarps][TC];
+  if constexpr (K::COLOUT) {  // NCT column tiles per block for these kinds
+    __shared__ T sm[kWarps][NCT * TC];
 #pragma unroll
-    for (int u = 0; u < CU; ++u)
+    for (int c = 0; c < NCT; ++c)
 #pragma unroll
-      for (int e = 0; e < V; ++e) {
-        const T s = cross_group_sum<LPR>(colacc[u][e]);
-        if (g == 0) sm[warp][(u * LPR + q) * V + e] = s;
-      }
+      for (int u = 0; u < CU; ++u)
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          const T s = cross_group_sum<LPR>(colacc[c][u][e]);
+          if (g == 0) sm[warp][c * TC + (u * LPR + q) * V + e] = s;
+        }
     __syncthreads();
-    for (int t = threadIdx.x; t < TC; t += kThreads) {
+    for (int t = threadIdx.x; t < NCT * TC; t += kThreads) {
       const int64_t j = c_lo + t;
       if (j >= p.cols) break;
       T s = sm[0][t];
@@ -283,7 +300,8 @@ __global__ void __launch_bounds__(kThreads) l2_finalize(const L2Args<T> p, int R
       }
     }
     if (K::COLOUT) {
-      const int64_t c_lo = (i / TC) * TC, c_hi = min(p.cols, c_lo + TC);
+      const int64_t span = (int64_t)TC * p.ctiles_per_cta;  // columns of one block
+      const int64_t c_lo = (i / span) * span, c_hi = min(p.cols, c_lo + span);
       for (int64_t rs = slice; rs < p.nrs; rs += SLICES) {
         const int64_t r_begin = rs * p.rows_per_cta, r_end = min(p.rows, r_begin + p.rows_per_cta);
         if (region_active<K::TRI>(r_begin, r_end, c_lo, c_hi)) s += __ldcg(p.colpart + rs * p.cols + i);
@@ -340,7 +358,7 @@ static int l2_launch_shape(const Launch& l, L2Args<T> args, int64_t rows_per_cta
   constexpr int RB = S::RB;
   args.nct = (int)((args.cols + TC - 1) / TC);
   args.xc_vec = (K::ROWOUT && V > 1 && aligned_to(args.xc, 16)) ? (args.incxc == 1 ? 1 : args.incxc == 2 ? 2 : 0) : 0;
-  if (K::COLOUT) ctiles_per_cta = 1;
+  if (K::COLOUT) ctiles_per_cta = S::NCT;
   if (ctiles_per_cta < 1) ctiles_per_cta = 1;
   if (ctiles_per_cta > args.nct) ctiles_per_cta = args.nct;
   rows_per_cta = ((rows_per_cta + RB - 1) / RB) * RB;
@@ -375,7 +393,7 @@ static int l2_launch_shape(const Launch& l, L2Args<T> args, int64_t rows_per_cta
   if (!args.direct) {
     const int64_t nout = K::ROWOUT ? args.rows : args.cols;
     const int nparts = (K::ROWOUT ? args.ncs : 0) + (K::COLOUT ? args.nrs : 0);
-    if (nparts >= 96) launch_finalize<T, K, 32>(l, args, RB, TC, nout);
+    if (nparts >= 512) launch_finalize<T, K, 32>(l, args, RB, TC, nout);
     else if (nparts >= 12) launch_finalize<T, K, 8>(l, args, RB, TC, nout);
     else launch_finalize<T, K, 1>(l, args, RB, TC, nout);
     if (int st = check_launch()) return st;
