@@ -392,6 +392,27 @@ def reference_arm(args):
     }))
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (replicas run independently; a
+    variant's time for the job is the slowest replica's).  Identity without a process group."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.cpu().tolist()
+
+
+def aggregate(specs, med_ms, world, peak):
+    """Per-variant rows and the whole-job value (N replicas: N x the geomean rate)."""
+    rows = []
+    for sp, t in zip(specs, med_ms):
+        gbs = sp["touched"] / (t * 1e-3) / 1e9
+        rows.append({"name": sp["name"], "family": sp["family"], "ms": t, "gbs": gbs,
+                     "gbs_useful": sp["useful"] / (t * 1e-3) / 1e9, "frac": gbs / peak})
+    return rows, world * geomean([r["gbs"] for r in rows])
+
+
 # --------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -452,10 +473,7 @@ def main():
     for k in range(nv):
         ts = sorted(events[s][k][0].elapsed_time(events[s][k][1]) for s in range(args.steps))
         med.append(ts[len(ts) // 2])
-    times = torch.tensor(med + [total_ms], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    times = times.cpu().tolist()
+    times = max_over_ranks(med + [total_ms], device)
     med, total_ms = times[:-1], times[-1]
     if rank != 0:
         if world > 1:
@@ -463,12 +481,7 @@ def main():
         return
 
     peak, peak_src = peak_gbs()
-    rows = []
-    for sp, t in zip(wl.specs, med):
-        gbs = world * sp["touched"] / (t * 1e-3) / 1e9
-        rows.append({"name": sp["name"], "family": sp["family"], "ms": t, "gbs": gbs / world,
-                     "gbs_useful": sp["useful"] / (t * 1e-3) / 1e9, "frac": gbs / world / peak})
-    value = world * geomean([r["gbs"] for r in rows])
+    rows, value = aggregate(wl.specs, med, world, peak)
     fam = {}
     for sp, r in zip(wl.specs, rows):
         f = fam.setdefault(sp["family"], {"ms": 0.0, "bytes": 0, "launches": 0})
