@@ -20,11 +20,13 @@ constexpr int kWarps = kThreads / 32;
 //   word 0      : ticket counter of the level-1 reductions
 //   word 16     : ticket counter of trsv (next block-row to hand out)
 //   word 17     : trsv "blocks finished" counter
+//   word 19     : sub-block trsv: abort flag (stays up after a timeout until the workspace is reset)
 // Scratch (partials, trsv flags) starts at kCtlBytes.
 constexpr size_t kCtlBytes = 4096;
 constexpr int kCtlReduceTicket = 0;
 constexpr int kCtlTrsvTicket = 16;
 constexpr int kCtlTrsvDone = 17;
+constexpr int kCtlTrsvAbort = 19;  // sub-block trsv: raised when a bounded wait ran out
 
 // ---------------------------------------------------------------------------------------
 // 16-byte packs: 4 floats or 2 doubles.
@@ -193,6 +195,7 @@ enum Knob {
   kKnobTrsvDebugSkip = 6,  // test hook: solve-order block that never publishes (-1 = none)
   kKnobTriWide = 7,
   kKnobTrsvPrefetchBytes = 8,  // total L2 bytes trsv blocks may prefetch ahead of the front
+  kKnobTrsvFront = 9,          // 1: sub-block trsv kernel where its preconditions hold; 0: general block-row kernel
   kKnobCount = 16
 };
 int64_t knob(int id);

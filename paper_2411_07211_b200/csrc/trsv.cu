@@ -31,6 +31,7 @@
 #include <atomic>
 
 #include "common.cuh"
+#include "trsv_front.cuh"
 
 namespace b2 {
 
@@ -567,6 +568,17 @@ static int trsv_impl(const b2_ctx* ctx, int order, int uplo, int trans, int diag
   Launch l;
   if (int st = make_launch(ctx, &l)) return st;
   if (n == 0) return B2_STATUS_OK;
+  // op(A) lower triangular <=> forward substitution
+  const bool eff_lower = (uplo == B2_LOWER) != (trans == B2_TRANS);
+  // rows of op(A) contiguous in memory <=> row-major N or column-major T
+  const bool coltype = (order == B2_ROW_MAJOR) != (trans == B2_NO_TRANS);
+  const bool unit = diag == B2_UNIT;
+  const unsigned tag = next_tag();
+  {
+    bool handled = false;
+    const int st = trsv_front_try<T>(l, coltype, !eff_lower, unit, n, a, lda, vec_base(x, n, incx), incx, tag, &handled);
+    if (handled) return st;
+  }
   constexpr int NB = trsv_block<T>();
   if ((n + NB - 1) / NB > 0x3fffffff) return B2_STATUS_NOT_IMPLEMENTED;
   const size_t xbuf_bytes = (size_t)n * 8 * (sizeof(T) / 4);
@@ -581,7 +593,7 @@ static int trsv_impl(const b2_ctx* ctx, int order, int uplo, int trans, int diag
   args.ticket = l.ctl + kCtlTrsvTicket;
   args.nb = (int)((n + NB - 1) / NB);
   args.nsb = (int)((n + kSB - 1) / kSB);
-  args.tag = next_tag();
+  args.tag = tag;
   args.wait_limit = l.wait_limit;
   args.device_status = l.device_status;
   args.debug_skip = (int)knob(kKnobTrsvDebugSkip);
@@ -590,11 +602,6 @@ static int trsv_impl(const b2_ctx* ctx, int order, int uplo, int trans, int diag
     int64_t d = knob(kKnobTrsvPrefetchBytes) / (tile_bytes * args.nb);
     args.pf_dist = (int)(d < 0 ? 0 : d > 64 ? 64 : d);
   }
-  // op(A) lower triangular <=> forward substitution
-  const bool eff_lower = (uplo == B2_LOWER) != (trans == B2_TRANS);
-  // rows of op(A) contiguous in memory <=> row-major N or column-major T
-  const bool coltype = (order == B2_ROW_MAJOR) != (trans == B2_NO_TRANS);
-  const bool unit = diag == B2_UNIT;
   constexpr int V = VecLen<T>::value;
   if (aligned_to(a, 16) && lda % V == 0) return trsv_variant<T, V>(l, args, coltype, !eff_lower, unit);
   return trsv_variant<T, 1>(l, args, coltype, !eff_lower, unit);

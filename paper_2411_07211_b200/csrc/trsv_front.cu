@@ -1,0 +1,577 @@
+// trsv, sub-block kernel: solve op(A) x = b in place (Section 6.2.2; same option space as trmv).
+//
+// The unknowns are cut into blocks of NB (128 float / 64 double).  In solve order (top-down for
+// an effectively lower-triangular op(A), bottom-up for an upper one) block row k needs
+//     x_k = inv(D_k) * (b_k - sum_{s<k} A_ks x_s),
+// and the chain k-1 -> k is the only sequential part.  Persistent 256-thread blocks draw block
+// rows in solve order.  A block
+//   1. inverts its diagonal block D_k in shared memory long before the front arrives
+//      (recursive doubling on 4x4 register tiles; the matrix is kept in symmetric storage so
+//      that both operand orientations are contiguous) and keeps inv(D_k) in registers,
+//   2. walks along its block row: tile A_ks sits in registers, distributed over a 16 x 16
+//      thread grid (an RS x RS sub-block per thread), so a tile-times-vector product needs RS
+//      vector elements per thread from shared memory and one RS-value reduction over the 16
+//      lanes of a row group -- a few hundred cycles from "x_s is here" to "row sums updated",
+//   3. treats inv(D_k) as one more tile whose vector is r = b - sum: the last trip through the
+//      SAME loop body produces x_k.  That matters: a stretch of code that a block executes
+//      once, after tens of microseconds of doing something else, costs microseconds of
+//      instruction fetches on the critical path; everything between "x_{k-1} is visible" and
+//      "x_k is published" is therefore code the block has been executing on every tile,
+//      including the publishing stores (earlier trips aim them at a dump area).
+// Values cross SMs as 64-bit words {32 payload bits, 32-bit call tag}: data and ready flag
+// are one store, and the consumer polls the data itself.  Every wait is bounded: when a
+// budget runs out the thread records B2_STATUS_TIMEOUT, raises an abort word in the control
+// block and every block drains without publishing.  Tickets are drawn in solve order, so a
+// block only waits for rows that running or finished blocks hold.
+#include "trsv_front.cuh"
+
+namespace b2 {
+namespace tf {
+
+constexpr int kT = 256;  // threads per block: a 16 x 16 grid of sub-block owners
+constexpr int kBar = 1;
+
+template <typename T>
+struct Geo;
+template <>
+struct Geo<float> {
+  static constexpr int NB = 128, V = 4;
+};
+template <>
+struct Geo<double> {
+  static constexpr int NB = 64, V = 2;
+};
+
+template <typename T>
+struct FrontArgs {
+  const T* a;
+  int64_t lda, n;
+  T* x;
+  int64_t incx;
+  unsigned long long* xbuf;  // solved x: WPE tagged words per unknown, padded to whole blocks
+  unsigned long long* dump;  // per block 2 * NB * WPE words nobody reads (stores of the non-final trips)
+  unsigned* ctl;
+  int nb;
+  int pf_dist;  // tiles pulled into L2 ahead of use
+  unsigned tag;
+  unsigned long long wait_limit;
+  int* device_status;
+  int debug_skip;
+};
+
+// ---------------------------------------------------------------------------------------
+// Named barrier.  Polling loops in front of it let lanes leave at different iterations, so the
+// warp is re-converged first and the form that counts threads (not whole warps) is used.
+__device__ __forceinline__ void bar_sync(int id, int count) {
+  __syncwarp();
+  asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void ld_word2(const unsigned long long* p, unsigned long long& a, unsigned long long& b) {
+  asm volatile("ld.relaxed.gpu.global.v2.u64 {%0,%1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void st_word(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned ld_flag(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+template <typename T>
+struct Words {
+  static constexpr int N = sizeof(T) / 4;
+};
+__device__ __forceinline__ void publish(unsigned long long* w, float v, unsigned tag) {
+  st_word(w, ((unsigned long long)tag << 32) | __float_as_uint(v));
+}
+__device__ __forceinline__ void publish(unsigned long long* w, double v, unsigned tag) {
+  const unsigned long long b = (unsigned long long)__double_as_longlong(v);
+  st_word(w, ((unsigned long long)tag << 32) | (b & 0xffffffffull));
+  st_word(w + 1, ((unsigned long long)tag << 32) | (b >> 32));
+}
+__device__ __forceinline__ float decode(const unsigned long long* w, float) { return __uint_as_float((unsigned)w[0]); }
+__device__ __forceinline__ double decode(const unsigned long long* w, double) {
+  return __longlong_as_double((long long)(((unsigned long long)(unsigned)w[1] << 32) | (unsigned)w[0]));
+}
+
+// Per-thread state of the bounded waits.
+struct Waiter {
+  unsigned long long budget;
+  unsigned tag;
+  unsigned* abort_word;  // control block: raised by the first wait that runs out
+  int* device_status;
+  bool dead;             // this thread stopped waiting (its budget ran out, or the abort word is up)
+
+  __device__ __forceinline__ void fail() {
+    dead = true;
+    atomicExch(abort_word, 1u);
+    if (device_status) atomicExch(device_status, (int)B2_STATUS_TIMEOUT);
+  }
+  // w holds a first attempt at the four words ptr[0..3] (16-byte aligned); polls until the
+  // words with their bit in `need` set carry this call's tag.
+  __device__ __forceinline__ void finish(unsigned long long (&w)[4], const unsigned long long* ptr, unsigned need,
+                                         unsigned sleep_ns) {
+    if (need == 0u) return;
+    for (;;) {
+      bool ok = true;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) ok = ok && (!((need >> i) & 1u) || (unsigned)(w[i] >> 32) == tag);
+      if (ok || dead) return;
+      if (--budget == 0) {
+        fail();
+        return;
+      }
+      if ((budget & 15) == 0 && ld_flag(abort_word) != 0u) {
+        dead = true;
+        return;
+      }
+      if (sleep_ns) __nanosleep(sleep_ns);
+      ld_word2(ptr, w[0], w[1]);
+      ld_word2(ptr + 2, w[2], w[3]);
+    }
+  }
+};
+
+// Four consecutive elements through 16-byte shared-memory accesses.
+__device__ __forceinline__ void ld4(const float* p, float (&v)[4]) {
+  const float4 t = *reinterpret_cast<const float4*>(p);
+  v[0] = t.x, v[1] = t.y, v[2] = t.z, v[3] = t.w;
+}
+__device__ __forceinline__ void ld4(const double* p, double (&v)[4]) {
+  const double2 t0 = *reinterpret_cast<const double2*>(p), t1 = *reinterpret_cast<const double2*>(p + 2);
+  v[0] = t0.x, v[1] = t0.y, v[2] = t1.x, v[3] = t1.y;
+}
+__device__ __forceinline__ void st4(float* p, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void st4(double* p, double a, double b, double c, double d) {
+  *reinterpret_cast<double2*>(p) = make_double2(a, b);
+  *reinterpret_cast<double2*>(p + 2) = make_double2(c, d);
+}
+
+// ---------------------------------------------------------------------------------------
+// COLTYPE: op(A)'s rows are columns of the stored row-major view.  BACKWARD: solve bottom-up.
+template <typename T, bool COLTYPE, bool BACKWARD, bool UNIT>
+__global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p) {
+  constexpr int NB = Geo<T>::NB, V = Geo<T>::V, WPE = Words<T>::N;
+  constexpr int RS = NB / 16;  // sub-block edge: 8 (float) / 4 (double)
+  constexpr int E = RS * RS;
+  constexpr int LPO = 16 / RS;                  // lanes per row owner
+  constexpr int SP = NB + 16 / (int)sizeof(T);  // row pitch of S (rows start 16-byte aligned)
+  constexpr bool CANON_LOWER = (COLTYPE == BACKWARD);  // stored triangle in the row-major view
+  using P = Pack<T, V>;
+
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  T* S = reinterpret_cast<T*>(smem_raw);       // diagonal block, then its inverse (symmetric storage)
+  T* Tm = S + NB * SP;                          // products in flight during the inversion
+  T* xs = Tm + (NB / 2) * (NB / 2 + 4);         // [2][NB] x values of the current / next tile
+  T* rbuf = xs + 2 * NB;                        // r = b - sum, the vector of the final trip
+  T* bvec = rbuf + NB;
+  __shared__ unsigned s_ticket[2];
+
+  const int ct = (int)threadIdx.x, warp = ct >> 5, lane = ct & 31;
+  const int rg = ct >> 4, cg = ct & 15;
+  const int ti = rg * RS + cg / LPO;  // the row (solve order inside the block) this thread may own
+  const bool owner = (cg % LPO) == 0;
+  unsigned long long* const dump = p.dump + (size_t)blockIdx.x * 2 * NB * WPE;
+
+  Waiter wt;
+  wt.budget = p.wait_limit ? p.wait_limit : (1ull << 22);
+  wt.tag = p.tag;
+  wt.abort_word = p.ctl + kCtlTrsvAbort;
+  wt.device_status = p.device_status;
+  wt.dead = false;
+  int parity = 0;
+
+  for (;;) {
+    if (ct == 0) {
+      unsigned kk = 0xffffffffu;
+      if (!wt.dead && ld_flag(wt.abort_word) == 0u) kk = atomicAdd(p.ctl + kCtlTrsvTicket, 1u);
+      s_ticket[parity] = kk;
+    }
+    bar_sync(kBar, kT);
+    const unsigned kk = s_ticket[parity];
+    parity ^= 1;
+    if (kk >= (unsigned)p.nb) break;
+    const int k = (int)kk;  // position in the solve order = number of source tiles
+    const int I = BACKWARD ? p.nb - 1 - k : k;
+    const int64_t r0 = (int64_t)I * NB;
+    const int nbI = (int)min((int64_t)NB, p.n - r0);
+    auto sidx = [&](int i) { return BACKWARD ? nbI - 1 - i : i; };  // solve order <-> memory order (involution)
+    auto blk = [&](int s) { return BACKWARD ? p.nb - 1 - s : s; };
+    const bool row_ok = ti < nbI;
+    const int mi = row_ok ? sidx(ti) : 0;  // memory-local row of this thread's unknown
+
+    // tile s of this block row -> registers: m[a * RS + b] = op(A)(row rg*RS + a, column cg*RS + b)
+    auto load_tile = [&](T (&m)[E], int s) {
+      const int64_t c0 = (int64_t)blk(s) * NB;
+      const int nbJ = (int)min((int64_t)NB, p.n - c0);
+      if (nbI == NB && nbJ == NB) {
+        // full tile: RS contiguous elements (32 bytes) per row of the sub-block in memory
+        const int64_t mr0 = BACKWARD ? NB - RS - rg * RS : rg * RS;  // memory-local first row of the sub-block
+#pragma unroll
+        for (int c = 0; c < RS; ++c) {
+          T v[RS];
+          const T* src = COLTYPE ? p.a + (c0 + cg * RS + c) * p.lda + r0 + mr0
+                                 : p.a + (r0 + mr0 + c) * p.lda + c0 + cg * RS;
+#pragma unroll
+          for (int u = 0; u < RS / V; ++u) {
+            const P pk = ld_nc<T, V>(src + u * V);
+#pragma unroll
+            for (int e = 0; e < V; ++e) v[u * V + e] = pk.v[e];
+          }
+          if (COLTYPE) {  // v runs along the rows of op(A) (memory order), c is the column
+#pragma unroll
+            for (int a = 0; a < RS; ++a) m[a * RS + c] = v[BACKWARD ? RS - 1 - a : a];
+          } else {        // v runs along the columns, c is the memory row of the sub-block
+#pragma unroll
+            for (int bcol = 0; bcol < RS; ++bcol) m[(BACKWARD ? RS - 1 - c : c) * RS + bcol] = v[bcol];
+          }
+        }
+      } else {
+#pragma unroll
+        for (int a = 0; a < RS; ++a)
+#pragma unroll
+          for (int bcol = 0; bcol < RS; ++bcol) {
+            const int i = rg * RS + a, jc = cg * RS + bcol;
+            const bool ok = i < nbI && jc < nbJ;
+            const int64_t mrow = r0 + (ok ? sidx(i) : 0), mcol = c0 + jc;
+            m[a * RS + bcol] = ok ? __ldg(COLTYPE ? p.a + mcol * p.lda + mrow : p.a + mrow * p.lda + mcol) : T(0);
+          }
+      }
+    };
+    // One 128-byte line per thread and call: tile s towards L2 (full tiles only).
+    auto prefetch_tile = [&](int s) {
+      if (s >= k || nbI < NB) return;
+      const int64_t c0 = (int64_t)blk(s) * NB;
+      if (p.n - c0 < NB) return;
+      constexpr int LPR = NB * (int)sizeof(T) / 128;  // lines per tile row
+      for (int i = ct; i < NB * LPR; i += kT) {
+        const T* ptr = p.a + ((COLTYPE ? c0 : r0) + i / LPR) * p.lda + (COLTYPE ? r0 : c0) + (i % LPR) * (128 / (int)sizeof(T));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+      }
+    };
+
+    // --- diagonal block -> S, solve order, symmetric storage (S[t][t'] = S[t'][t]); b -> bvec
+    if (nbI < NB)
+      for (int idx = ct; idx < NB * SP; idx += kT) S[idx] = T(0);
+    if (ct < NB) {
+      const T bv = ct < nbI ? p.x[(r0 + sidx(ct)) * p.incx] : T(0);
+      bvec[ct] = bv;
+      rbuf[ct] = bv;  // r = b when nothing precedes
+    }
+    if (nbI < NB) bar_sync(kBar, kT);
+    {
+      constexpr int PACKS = NB * NB / V;
+      constexpr int PPT = PACKS / kT;  // packs per thread: 16 (float) / 8 (double)
+      P v[PPT];
+#pragma unroll
+      for (int m = 0; m < PPT; ++m) {
+        const int idx = m * kT + ct, pr = idx / (NB / V), pc = (idx % (NB / V)) * V;
+        const bool use = pr < nbI && pc < nbI && (CANON_LOWER ? pc <= pr : pc + V - 1 >= pr);  // pack touches the triangle
+        if (use && pc + V <= nbI) {
+          v[m] = ld_nc<T, V>(p.a + (r0 + pr) * p.lda + r0 + pc);
+        } else {
+#pragma unroll
+          for (int e = 0; e < V; ++e)
+            v[m].v[e] = (use && pc + e < nbI) ? __ldg(p.a + (r0 + pr) * p.lda + r0 + pc + e) : T(0);
+        }
+      }
+#pragma unroll
+      for (int m = 0; m < PPT; ++m) {
+        const int idx = m * kT + ct, pr = idx / (NB / V), pc0 = (idx % (NB / V)) * V;
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          const int pc = pc0 + e;
+          const bool in_tri = pr < nbI && pc < nbI && (CANON_LOWER ? pc <= pr : pc >= pr);
+          if (in_tri) {
+            const int sr = sidx(pr), sc = sidx(pc);
+            const T val = (pr == pc && UNIT) ? T(1) : v[m].v[e];
+            S[sr * SP + sc] = val;
+            S[sc * SP + sr] = val;
+          }
+        }
+      }
+    }
+    for (int s = ct; s < NB; s += kT)
+      if (s >= nbI) S[s * SP + s] = T(1);
+    for (int s = 0; s < p.pf_dist; ++s) prefetch_tile(s);
+    bar_sync(kBar, kT);
+
+    // --- in-place inverse.  4x4 diagonal blocks by substitution (one column per thread) ...
+    {
+      T col[4];
+      const int c = ct, d0 = (c / 4) * 4, lc = c % 4;
+      if (ct < NB) {
+        T e[4][4];
+#pragma unroll
+        for (int ls = 0; ls < 4; ++ls)
+#pragma unroll
+          for (int lt = 0; lt <= ls; ++lt) e[ls][lt] = S[(d0 + ls) * SP + d0 + lt];
+#pragma unroll
+        for (int ls = 0; ls < 4; ++ls) {
+          T acc = (ls == lc) ? T(1) : T(0);
+#pragma unroll
+          for (int lt = 0; lt < ls; ++lt) acc -= e[ls][lt] * col[lt];
+          col[ls] = acc / e[ls][ls];
+        }
+      }
+      bar_sync(kBar, kT);
+      if (ct < NB) {
+#pragma unroll
+        for (int ls = 0; ls < 4; ++ls)
+          if (ls >= lc) {
+            S[(d0 + ls) * SP + c] = col[ls];
+            S[c * SP + d0 + ls] = col[ls];
+          }
+      }
+      bar_sync(kBar, kT);
+    }
+    // ... then, for h = 4 .. NB/2, every pair [A 0; C B] of h x h blocks gets its lower-left
+    // block -inv(B) (C inv(A)).  Left operands are read through the mirrored half of S.
+#pragma unroll 1
+    for (int h = 4; h < NB; h *= 2) {
+      const int tpr = h / 4, per_pair = tpr * tpr, total = (NB / (2 * h)) * per_pair;
+      const int TP = h + 4;
+      for (int e = ct; e < total; e += kT) {  // Tm = C * inv(A); lanes along the rows of Tm
+        const int pr = e / per_pair, rem = e % per_pair, i0 = (rem % tpr) * 4, j0 = (rem / tpr) * 4;
+        const int top = pr * 2 * h, bot = top + h;
+        T acc[4][4];
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) acc[ii][jj] = T(0);
+#pragma unroll
+        for (int dl = 0; dl < 4; ++dl) {  // inv(A) is zero above its diagonal
+          const T* rowp = S + (top + j0 + dl) * SP;
+          T cv[4], av[4];
+          ld4(rowp + bot + i0, cv);
+          ld4(rowp + top + j0, av);
+#pragma unroll
+          for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+              if (jj <= dl) acc[ii][jj] = cv[ii] * av[jj] + acc[ii][jj];
+        }
+#pragma unroll 4
+        for (int l = j0 + 4; l < h; ++l) {
+          const T* rowp = S + (top + l) * SP;
+          T cv[4], av[4];
+          ld4(rowp + bot + i0, cv);
+          ld4(rowp + top + j0, av);
+#pragma unroll
+          for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) acc[ii][jj] = cv[ii] * av[jj] + acc[ii][jj];
+        }
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii)
+          st4(Tm + (pr * h + i0 + ii) * TP + j0, acc[ii][0], acc[ii][1], acc[ii][2], acc[ii][3]);
+      }
+      bar_sync(kBar, kT);
+      for (int e = ct; e < total; e += kT) {  // X = -inv(B) * Tm; lanes along the columns of X
+        const int pr = e / per_pair, rem = e % per_pair, j0 = (rem % tpr) * 4, i0 = (rem / tpr) * 4;
+        const int top = pr * 2 * h, bot = top + h;
+        T acc[4][4];
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) acc[ii][jj] = T(0);
+#pragma unroll 4
+        for (int l = 0; l < i0; ++l) {
+          T bv[4], tv[4];
+          ld4(S + (bot + l) * SP + bot + i0, bv);
+          ld4(Tm + (pr * h + l) * TP + j0, tv);
+#pragma unroll
+          for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) acc[ii][jj] = bv[ii] * tv[jj] + acc[ii][jj];
+        }
+#pragma unroll
+        for (int dl = 0; dl < 4; ++dl) {  // inv(B) is zero above its diagonal
+          T bv[4], tv[4];
+          ld4(S + (bot + i0 + dl) * SP + bot + i0, bv);
+          ld4(Tm + (pr * h + i0 + dl) * TP + j0, tv);
+#pragma unroll
+          for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+              if (ii >= dl) acc[ii][jj] = bv[ii] * tv[jj] + acc[ii][jj];
+        }
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii)
+          st4(S + (bot + i0 + ii) * SP + top + j0, -acc[ii][0], -acc[ii][1], -acc[ii][2], -acc[ii][3]);
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj)
+          st4(S + (top + j0 + jj) * SP + bot + i0, -acc[0][jj], -acc[1][jj], -acc[2][jj], -acc[3][jj]);
+      }
+      bar_sync(kBar, kT);
+    }
+    // --- this thread's sub-block of the inverse -> registers (zero above the diagonal)
+    T winv[E];
+#pragma unroll
+    for (int a = 0; a < RS; ++a)
+#pragma unroll
+      for (int u = 0; u < RS / 4; ++u) {
+        T v4[4];
+        ld4(S + (rg * RS + a) * SP + cg * RS + u * 4, v4);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) winv[a * RS + u * 4 + e] = (cg * RS + u * 4 + e <= rg * RS + a) ? v4[e] : T(0);
+      }
+
+    // --- along the block row; trip `k` (the last) applies the inverse
+    T cur[E];
+    if (k > 0) load_tile(cur, 0);
+    const T bi = bvec[ti];
+    T racc = T(0);
+    // warp 0 fetches the x values of a tile: 4 tagged words per lane, first attempt one trip ahead
+    unsigned long long xw[4] = {0, 0, 0, 0};
+    unsigned xneed = 0;
+    const unsigned long long* xptr = p.xbuf;
+    auto x_issue = [&](int s) {
+      const int64_t xi = (int64_t)blk(s) * NB + V * lane;
+      xneed = 0;
+#pragma unroll
+      for (int e = 0; e < V; ++e)
+        if (xi + e < p.n) xneed |= ((1u << WPE) - 1u) << (e * WPE);
+      xptr = p.xbuf + xi * WPE;
+      if (xneed) {
+        ld_word2(xptr, xw[0], xw[1]);
+        ld_word2(xptr + 2, xw[2], xw[3]);
+      }
+    };
+    if (warp == 0 && k > 0) x_issue(0);
+
+    int ntrips = k + 1;
+    asm volatile("" : "+r"(ntrips));  // one loop, not a peeled copy of its last trip
+#pragma unroll 1
+    for (int it = 0; it < ntrips; ++it) {
+      const bool last = it == k;
+      T* xbuf_s = xs + (it & 1) * NB;
+      if (warp == 0 && !last) {
+        const int dist = k - it;  // rows between this block and the producer of the tile's x
+        wt.finish(xw, xptr, xneed, dist > 2 ? (unsigned)min((dist - 2) * 200, 2000) : 0u);
+        P xv;
+#pragma unroll
+        for (int e = 0; e < V; ++e) xv.v[e] = ((xneed >> (e * WPE)) & 1u) ? decode(xw + e * WPE, T(0)) : T(0);
+        *reinterpret_cast<P*>(xbuf_s + V * lane) = xv;
+      }
+      bar_sync(kBar, kT);
+      if (warp == 0 && it + 1 < k) x_issue(it + 1);
+      const T* vec = last ? rbuf : xbuf_s;
+      T xv[RS], part[RS];
+#pragma unroll
+      for (int u = 0; u < RS / 4; ++u) {
+        T v4[4];
+        ld4(vec + cg * RS + u * 4, v4);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) xv[u * 4 + e] = v4[e];
+      }
+#pragma unroll
+      for (int a = 0; a < RS; ++a) {
+        part[a] = T(0);
+#pragma unroll
+        for (int bcol = 0; bcol < RS; ++bcol)
+          part[a] = (last ? winv[a * RS + bcol] : cur[a * RS + bcol]) * xv[bcol] + part[a];
+      }
+      if (it + 1 < k) load_tile(cur, it + 1);
+      const T s = multi_group_sum<16, RS>(part, lane);
+      if (!last) racc += s;
+      if (owner && !last) rbuf[ti] = bi - racc;
+      if (owner && row_ok && !wt.dead) {
+        // every trip stores; only the last one aims at the real destinations
+        const bool real = last && k != p.debug_skip;
+        unsigned long long* dw = real ? p.xbuf + (r0 + mi) * WPE : dump + ti * WPE;
+        T* dx = real ? p.x + (r0 + mi) * p.incx : reinterpret_cast<T*>(dump + NB * WPE) + ti;
+        publish(dw, s, real ? p.tag : 0u);
+        *dx = s;
+      }
+      prefetch_tile(it + 1 + p.pf_dist);
+    }
+    bar_sync(kBar, kT);  // S, bvec, rbuf, xs are reused by the next block row
+  }
+  // The last block out leaves the control block clean (not after an abort: the caller resets).
+  if (ct == 0 && ld_flag(p.ctl + kCtlTrsvAbort) == 0u) {
+    __threadfence();
+    const unsigned d = atomicAdd(p.ctl + kCtlTrsvDone, 1u);
+    if (d == gridDim.x - 1) {
+      p.ctl[kCtlTrsvTicket] = 0u;
+      p.ctl[kCtlTrsvDone] = 0u;
+    }
+  }
+}
+
+template <typename T>
+constexpr size_t front_smem_bytes() {
+  constexpr int NB = Geo<T>::NB;
+  constexpr int SP = NB + 16 / (int)sizeof(T);
+  return sizeof(T) * (size_t)(NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB);
+}
+
+template <typename T, bool COLTYPE, bool BACKWARD, bool UNIT>
+static int launch_one(const Launch& l, const FrontArgs<T>& args, int grid) {
+  constexpr size_t smem = front_smem_bytes<T>();
+  auto kern = trsv_front_kernel<T, COLTYPE, BACKWARD, UNIT>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return B2_STATUS_LAUNCH_FAILED;
+  }
+  kern<<<grid, kT, smem, l.stream>>>(args);
+  return check_launch();
+}
+
+template <typename T, bool COLTYPE, bool BACKWARD>
+static int launch_diag(const Launch& l, const FrontArgs<T>& args, int grid, bool unit) {
+  return unit ? launch_one<T, COLTYPE, BACKWARD, true>(l, args, grid)
+              : launch_one<T, COLTYPE, BACKWARD, false>(l, args, grid);
+}
+
+}  // namespace tf
+
+template <typename T>
+int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int64_t n, const T* a, int64_t lda,
+                   T* xbase, int64_t incx, unsigned tag, bool* handled) {
+  using namespace tf;
+  constexpr int NB = Geo<T>::NB, V = Geo<T>::V, WPE = Words<T>::N;
+  *handled = false;
+  if (!knob(kKnobTrsvFront)) return B2_STATUS_OK;
+  if (!aligned_to(a, 16) || lda % V != 0) return B2_STATUS_OK;
+  const int64_t nb64 = (n + NB - 1) / NB;
+  if (nb64 > 0x3fffffff) return B2_STATUS_OK;
+  const int nb = (int)nb64;
+  const int grid = nb < sm_count() ? nb : sm_count();
+  const size_t xbuf_words = (size_t)nb * NB * WPE;
+  const size_t dump_words = (size_t)grid * 2 * NB * WPE;
+  if ((xbuf_words + dump_words) * 8 > l.scratch_bytes) return B2_STATUS_OK;
+  FrontArgs<T> args = {};
+  args.a = a;
+  args.lda = lda;
+  args.n = n;
+  args.x = xbase;
+  args.incx = incx;
+  args.xbuf = reinterpret_cast<unsigned long long*>(l.scratch);
+  args.dump = args.xbuf + xbuf_words;
+  args.ctl = l.ctl;
+  args.nb = nb;
+  {  // keep the prefetched-but-unused tiles of all blocks within a fraction of L2
+    const int64_t tile_bytes = (int64_t)NB * NB * sizeof(T);
+    int64_t d = knob(kKnobTrsvPrefetchBytes) / (tile_bytes * grid);
+    args.pf_dist = (int)(d < 0 ? 0 : d > 16 ? 16 : d);
+  }
+  args.tag = tag;
+  args.wait_limit = l.wait_limit;
+  args.device_status = l.device_status;
+  args.debug_skip = (int)knob(kKnobTrsvDebugSkip);
+  *handled = true;
+  if (coltype)
+    return backward ? launch_diag<T, true, true>(l, args, grid, unit) : launch_diag<T, true, false>(l, args, grid, unit);
+  return backward ? launch_diag<T, false, true>(l, args, grid, unit) : launch_diag<T, false, false>(l, args, grid, unit);
+}
+
+template int trsv_front_try<float>(const Launch&, bool, bool, bool, int64_t, const float*, int64_t, float*, int64_t,
+                                   unsigned, bool*);
+template int trsv_front_try<double>(const Launch&, bool, bool, bool, int64_t, const double*, int64_t, double*, int64_t,
+                                    unsigned, bool*);
+
+}  // namespace b2
