@@ -13,7 +13,7 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobTrsvDebugSkip   */ -1,
     /* kKnobTriWide         */ 0,
     /* kKnobTrsvPrefetchBytes */ 48 << 20,
-    /* kKnobTrsvFront       */ 0,
+    /* kKnobTrsvFront       */ 1,
 };
 
 unsigned long long g_launch_count = 0;

@@ -17,7 +17,7 @@
 //      once, after tens of microseconds of doing something else, costs microseconds of
 //      instruction fetches on the critical path; everything between "x_{k-1} is visible" and
 //      "x_k is published" is therefore code the block has been executing on every tile,
-//      including the publishing stores (earlier trips aim them at a dump area).
+//      including the publishing stores (predicated off on the earlier trips).
 // Values cross SMs as 64-bit words {32 payload bits, 32-bit call tag}: data and ready flag
 // are one store, and the consumer polls the data itself.  Every wait is bounded: when a
 // budget runs out the thread records B2_STATUS_TIMEOUT, raises an abort word in the control
@@ -49,7 +49,6 @@ struct FrontArgs {
   T* x;
   int64_t incx;
   unsigned long long* xbuf;  // solved x: WPE tagged words per unknown, padded to whole blocks
-  unsigned long long* dump;  // per block 2 * NB * WPE words nobody reads (stores of the non-final trips)
   unsigned* ctl;
   int nb;
   int pf_dist;  // tiles pulled into L2 ahead of use
@@ -57,7 +56,22 @@ struct FrontArgs {
   unsigned long long wait_limit;
   int* device_status;
   int debug_skip;
+#ifdef B2_TRSV_TRACE
+  unsigned long long* trace;  // [nb][16] time stamps (ns)
+#endif
 };
+
+#ifdef B2_TRSV_TRACE
+__device__ __forceinline__ unsigned long long now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// stamps go to shared memory and are flushed after the row is published
+#define B2_CTRACE(cond, slot) do { if (cond) s_trace[slot] = now_ns(); } while (0)
+#else
+#define B2_CTRACE(cond, slot) do { } while (0)
+#endif
 
 // ---------------------------------------------------------------------------------------
 // Named barrier.  Polling loops in front of it let lanes leave at different iterations, so the
@@ -69,8 +83,20 @@ __device__ __forceinline__ void bar_sync(int id, int count) {
 __device__ __forceinline__ void ld_word2(const unsigned long long* p, unsigned long long& a, unsigned long long& b) {
   asm volatile("ld.relaxed.gpu.global.v2.u64 {%0,%1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
 }
-__device__ __forceinline__ void st_word(unsigned long long* p, unsigned long long v) {
-  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+// Stores under a predicate instead of a branch: the instructions are fetched on every trip of
+// the tile loop and take effect on the last one only.
+__device__ __forceinline__ void st_word_if(bool pred, unsigned long long* p, unsigned long long v) {
+  asm volatile("{ .reg .pred q; setp.ne.u32 q, %0, 0; @q st.relaxed.gpu.global.u64 [%1], %2; }" ::"r"((unsigned)pred),
+               "l"(p), "l"(v)
+               : "memory");
+}
+__device__ __forceinline__ void st_val_if(bool pred, float* p, float v) {
+  asm volatile("{ .reg .pred q; setp.ne.u32 q, %0, 0; @q st.global.f32 [%1], %2; }" ::"r"((unsigned)pred), "l"(p), "f"(v)
+               : "memory");
+}
+__device__ __forceinline__ void st_val_if(bool pred, double* p, double v) {
+  asm volatile("{ .reg .pred q; setp.ne.u32 q, %0, 0; @q st.global.f64 [%1], %2; }" ::"r"((unsigned)pred), "l"(p), "d"(v)
+               : "memory");
 }
 __device__ __forceinline__ unsigned ld_flag(const unsigned* p) {
   unsigned v;
@@ -82,13 +108,13 @@ template <typename T>
 struct Words {
   static constexpr int N = sizeof(T) / 4;
 };
-__device__ __forceinline__ void publish(unsigned long long* w, float v, unsigned tag) {
-  st_word(w, ((unsigned long long)tag << 32) | __float_as_uint(v));
+__device__ __forceinline__ void publish_if(bool pred, unsigned long long* w, float v, unsigned tag) {
+  st_word_if(pred, w, ((unsigned long long)tag << 32) | __float_as_uint(v));
 }
-__device__ __forceinline__ void publish(unsigned long long* w, double v, unsigned tag) {
+__device__ __forceinline__ void publish_if(bool pred, unsigned long long* w, double v, unsigned tag) {
   const unsigned long long b = (unsigned long long)__double_as_longlong(v);
-  st_word(w, ((unsigned long long)tag << 32) | (b & 0xffffffffull));
-  st_word(w + 1, ((unsigned long long)tag << 32) | (b >> 32));
+  st_word_if(pred, w, ((unsigned long long)tag << 32) | (b & 0xffffffffull));
+  st_word_if(pred, w + 1, ((unsigned long long)tag << 32) | (b >> 32));
 }
 __device__ __forceinline__ float decode(const unsigned long long* w, float) { return __uint_as_float((unsigned)w[0]); }
 __device__ __forceinline__ double decode(const unsigned long long* w, double) {
@@ -133,6 +159,16 @@ struct Waiter {
   }
 };
 
+// 16-byte load through a generic address (global memory or shared memory), issued where it
+// stands: the compiler must not sink it towards its first use.
+template <typename T, int N>
+__device__ __forceinline__ Pack<T, N> ld_generic(const T* p) {
+  static_assert(sizeof(T) * N == 16, "16-byte packs");
+  uint4 t;
+  asm volatile("ld.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(t.x), "=r"(t.y), "=r"(t.z), "=r"(t.w) : "l"(p) : "memory");
+  return *reinterpret_cast<Pack<T, N>*>(&t);
+}
+
 // Four consecutive elements through 16-byte shared-memory accesses.
 __device__ __forceinline__ void ld4(const float* p, float (&v)[4]) {
   const float4 t = *reinterpret_cast<const float4*>(p);
@@ -158,6 +194,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
   constexpr int RS = NB / 16;  // sub-block edge: 8 (float) / 4 (double)
   constexpr int E = RS * RS;
   constexpr int LPO = 16 / RS;                  // lanes per row owner
+  constexpr int H = NB / 2;                     // distance between a thread's two chunks
   constexpr int SP = NB + 16 / (int)sizeof(T);  // row pitch of S (rows start 16-byte aligned)
   constexpr bool CANON_LOWER = (COLTYPE == BACKWARD);  // stored triangle in the row-major view
   using P = Pack<T, V>;
@@ -165,16 +202,20 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* S = reinterpret_cast<T*>(smem_raw);       // diagonal block, then its inverse (symmetric storage)
   T* Tm = S + NB * SP;                          // products in flight during the inversion
-  T* xs = Tm + (NB / 2) * (NB / 2 + 4);         // [2][NB] x values of the current / next tile
+  T* Wt = Tm + (NB / 2) * (NB / 2 + 4);         // the finished inverse in the tile loader's layout
+  T* xs = Wt + NB * SP;                         // [2][NB] x values of the current / next tile
   T* rbuf = xs + 2 * NB;                        // r = b - sum, the vector of the final trip
   T* bvec = rbuf + NB;
   __shared__ unsigned s_ticket[2];
+#ifdef B2_TRSV_TRACE
+  __shared__ unsigned long long s_trace[16];
+#endif
 
   const int ct = (int)threadIdx.x, warp = ct >> 5, lane = ct & 31;
   const int rg = ct >> 4, cg = ct & 15;
-  const int ti = rg * RS + cg / LPO;  // the row (solve order inside the block) this thread may own
+  // the row (solve order inside the block) this thread may own: sub-block row a = cg / LPO
+  const int ti = ((cg / LPO) / V) * H + V * rg + ((cg / LPO) % V);
   const bool owner = (cg % LPO) == 0;
-  unsigned long long* const dump = p.dump + (size_t)blockIdx.x * 2 * NB * WPE;
 
   Waiter wt;
   wt.budget = p.wait_limit ? p.wait_limit : (1ull << 22);
@@ -195,6 +236,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     parity ^= 1;
     if (kk >= (unsigned)p.nb) break;
     const int k = (int)kk;  // position in the solve order = number of source tiles
+    B2_CTRACE(ct == 0, 0);
     const int I = BACKWARD ? p.nb - 1 - k : k;
     const int64_t r0 = (int64_t)I * NB;
     const int nbI = (int)min((int64_t)NB, p.n - r0);
@@ -203,41 +245,53 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     const bool row_ok = ti < nbI;
     const int mi = row_ok ? sidx(ti) : 0;  // memory-local row of this thread's unknown
 
-    // tile s of this block row -> registers: m[a * RS + b] = op(A)(row rg*RS + a, column cg*RS + b)
+    // tile s of this block row -> registers: m[a * RS + b] = op(A)(row sub_i(a), column sub_j(b)).
+    // A thread's RS rows / columns are two chunks of V (one 16-byte pack), NB/2 apart: the packs
+    // that the lanes of a warp load together then tile whole 32-byte sectors.
+    // "Tile" k is the inverse of the diagonal block, laid out in shared memory (Wt) so that the
+    // very same loads fetch it: the addresses are generic.
     auto load_tile = [&](T (&m)[E], int s) {
-      const int64_t c0 = (int64_t)blk(s) * NB;
-      const int nbJ = (int)min((int64_t)NB, p.n - c0);
-      if (nbI == NB && nbJ == NB) {
-        // full tile: RS contiguous elements (32 bytes) per row of the sub-block in memory
-        const int64_t mr0 = BACKWARD ? NB - RS - rg * RS : rg * RS;  // memory-local first row of the sub-block
+      const bool inv = s == k;
+      const int64_t c0 = inv ? 0 : (int64_t)blk(s) * NB;
+      const int nbJ = inv ? NB : (int)min((int64_t)NB, p.n - c0);
+      if (inv || (nbI == NB && nbJ == NB)) {
+        const T* base = inv ? Wt : p.a;
+        const int64_t ld = inv ? SP : p.lda, rr0 = inv ? 0 : r0;
+        if (!COLTYPE) {
 #pragma unroll
-        for (int c = 0; c < RS; ++c) {
-          T v[RS];
-          const T* src = COLTYPE ? p.a + (c0 + cg * RS + c) * p.lda + r0 + mr0
-                                 : p.a + (r0 + mr0 + c) * p.lda + c0 + cg * RS;
+          for (int a = 0; a < RS; ++a) {
+            const int i = (a / V) * H + V * rg + (a % V);
+            const T* src = base + (rr0 + (BACKWARD ? NB - 1 - i : i)) * ld + c0 + V * cg;
 #pragma unroll
-          for (int u = 0; u < RS / V; ++u) {
-            const P pk = ld_nc<T, V>(src + u * V);
+            for (int hb = 0; hb < RS / V; ++hb) {
+              const P pk = ld_generic<T, V>(src + hb * H);
 #pragma unroll
-            for (int e = 0; e < V; ++e) v[u * V + e] = pk.v[e];
+              for (int e = 0; e < V; ++e) m[a * RS + hb * V + e] = pk.v[e];
+            }
           }
-          if (COLTYPE) {  // v runs along the rows of op(A) (memory order), c is the column
+        } else {
 #pragma unroll
-            for (int a = 0; a < RS; ++a) m[a * RS + c] = v[BACKWARD ? RS - 1 - a : a];
-          } else {        // v runs along the columns, c is the memory row of the sub-block
+          for (int b = 0; b < RS; ++b) {
+            const int j = (b / V) * H + V * cg + (b % V);
+            const T* src = base + (c0 + j) * ld + rr0;
 #pragma unroll
-            for (int bcol = 0; bcol < RS; ++bcol) m[(BACKWARD ? RS - 1 - c : c) * RS + bcol] = v[bcol];
+            for (int ha = 0; ha < RS / V; ++ha) {
+              const int m0 = BACKWARD ? NB - ha * H - V * rg - V : ha * H + V * rg;  // ascending memory run of the chunk
+              const P pk = ld_generic<T, V>(src + m0);
+#pragma unroll
+              for (int e = 0; e < V; ++e) m[(ha * V + (BACKWARD ? V - 1 - e : e)) * RS + b] = pk.v[e];
+            }
           }
         }
       } else {
 #pragma unroll
         for (int a = 0; a < RS; ++a)
 #pragma unroll
-          for (int bcol = 0; bcol < RS; ++bcol) {
-            const int i = rg * RS + a, jc = cg * RS + bcol;
+          for (int b = 0; b < RS; ++b) {
+            const int i = (a / V) * H + V * rg + (a % V), jc = (b / V) * H + V * cg + (b % V);
             const bool ok = i < nbI && jc < nbJ;
             const int64_t mrow = r0 + (ok ? sidx(i) : 0), mcol = c0 + jc;
-            m[a * RS + bcol] = ok ? __ldg(COLTYPE ? p.a + mcol * p.lda + mrow : p.a + mrow * p.lda + mcol) : T(0);
+            m[a * RS + b] = ok ? __ldg(COLTYPE ? p.a + mcol * p.lda + mrow : p.a + mrow * p.lda + mcol) : T(0);
           }
       }
     };
@@ -408,21 +462,19 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       }
       bar_sync(kBar, kT);
     }
-    // --- this thread's sub-block of the inverse -> registers (zero above the diagonal)
-    T winv[E];
-#pragma unroll
-    for (int a = 0; a < RS; ++a)
-#pragma unroll
-      for (int u = 0; u < RS / 4; ++u) {
-        T v4[4];
-        ld4(S + (rg * RS + a) * SP + cg * RS + u * 4, v4);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) winv[a * RS + u * 4 + e] = (cg * RS + u * 4 + e <= rg * RS + a) ? v4[e] : T(0);
-      }
+    // --- the inverse (zero above its diagonal) -> Wt, indexed the way load_tile reads a tile
+    for (int idx = ct; idx < NB * NB; idx += kT) {
+      const int rho = idx / NB, gam = idx % NB;
+      const int i = COLTYPE ? (BACKWARD ? NB - 1 - gam : gam) : (BACKWARD ? NB - 1 - rho : rho);
+      const int j = COLTYPE ? rho : gam;
+      Wt[rho * SP + gam] = j <= i ? S[i * SP + j] : T(0);
+    }
+    bar_sync(kBar, kT);
 
+    B2_CTRACE(ct == 0, 1);
     // --- along the block row; trip `k` (the last) applies the inverse
-    T cur[E];
-    if (k > 0) load_tile(cur, 0);
+    T cur[E], nxt[E];
+    load_tile(cur, 0);
     const T bi = bvec[ti];
     T racc = T(0);
     // warp 0 fetches the x values of a tile: 4 tagged words per lane, first attempt one trip ahead
@@ -449,47 +501,56 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     for (int it = 0; it < ntrips; ++it) {
       const bool last = it == k;
       T* xbuf_s = xs + (it & 1) * NB;
+      // first of all, off the critical path: the next tile (or the inverse) into the second
+      // register set and a tile further ahead towards L2 -- in flight while this trip waits
+      if (!last) load_tile(nxt, it + 1);
+      prefetch_tile(it + 1 + p.pf_dist);
       if (warp == 0 && !last) {
         const int dist = k - it;  // rows between this block and the producer of the tile's x
+        B2_CTRACE(ct == 0 && it == k - 1, 2);
         wt.finish(xw, xptr, xneed, dist > 2 ? (unsigned)min((dist - 2) * 200, 2000) : 0u);
+        B2_CTRACE(ct == 0 && it == k - 1, 3);
         P xv;
 #pragma unroll
         for (int e = 0; e < V; ++e) xv.v[e] = ((xneed >> (e * WPE)) & 1u) ? decode(xw + e * WPE, T(0)) : T(0);
         *reinterpret_cast<P*>(xbuf_s + V * lane) = xv;
       }
       bar_sync(kBar, kT);
-      if (warp == 0 && it + 1 < k) x_issue(it + 1);
+      B2_CTRACE(ct == 0 && it == k - 1, 8);
+      B2_CTRACE(ct == 0 && last, 9);
       const T* vec = last ? rbuf : xbuf_s;
       T xv[RS], part[RS];
 #pragma unroll
-      for (int u = 0; u < RS / 4; ++u) {
-        T v4[4];
-        ld4(vec + cg * RS + u * 4, v4);
+      for (int hb = 0; hb < RS / V; ++hb) {
+        const P pk = *reinterpret_cast<const P*>(vec + hb * H + V * cg);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) xv[u * 4 + e] = v4[e];
+        for (int e = 0; e < V; ++e) xv[hb * V + e] = pk.v[e];
       }
 #pragma unroll
       for (int a = 0; a < RS; ++a) {
         part[a] = T(0);
 #pragma unroll
-        for (int bcol = 0; bcol < RS; ++bcol)
-          part[a] = (last ? winv[a * RS + bcol] : cur[a * RS + bcol]) * xv[bcol] + part[a];
+        for (int bcol = 0; bcol < RS; ++bcol) part[a] = cur[a * RS + bcol] * xv[bcol] + part[a];
       }
-      if (it + 1 < k) load_tile(cur, it + 1);
       const T s = multi_group_sum<16, RS>(part, lane);
+      B2_CTRACE(ct == 0 && it == k - 1, 7);
+      B2_CTRACE(ct == 0 && last, 10);
       if (!last) racc += s;
       if (owner && !last) rbuf[ti] = bi - racc;
-      if (owner && row_ok && !wt.dead) {
-        // every trip stores; only the last one aims at the real destinations
-        const bool real = last && k != p.debug_skip;
-        unsigned long long* dw = real ? p.xbuf + (r0 + mi) * WPE : dump + ti * WPE;
-        T* dx = real ? p.x + (r0 + mi) * p.incx : reinterpret_cast<T*>(dump + NB * WPE) + ti;
-        publish(dw, s, real ? p.tag : 0u);
-        *dx = s;
+      {  // publishing stores: fetched on every trip, performed on the last
+        const bool real = last && owner && row_ok && !wt.dead && k != p.debug_skip;
+        publish_if(real, p.xbuf + (r0 + mi) * WPE, s, p.tag);
+        st_val_if(real, p.x + (r0 + mi) * p.incx, s);
       }
-      prefetch_tile(it + 1 + p.pf_dist);
+      B2_CTRACE(ct == 0 && last, 4);
+      if (warp == 0 && it + 1 < k) x_issue(it + 1);  // first attempt at the x words of the next tile
+#pragma unroll
+      for (int e = 0; e < E; ++e) cur[e] = nxt[e];
     }
     bar_sync(kBar, kT);  // S, bvec, rbuf, xs are reused by the next block row
+#ifdef B2_TRSV_TRACE
+    if (ct < 16) p.trace[k * 16 + ct] = s_trace[ct];
+#endif
   }
   // The last block out leaves the control block clean (not after an abort: the caller resets).
   if (ct == 0 && ld_flag(p.ctl + kCtlTrsvAbort) == 0u) {
@@ -506,7 +567,7 @@ template <typename T>
 constexpr size_t front_smem_bytes() {
   constexpr int NB = Geo<T>::NB;
   constexpr int SP = NB + 16 / (int)sizeof(T);
-  return sizeof(T) * (size_t)(NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB);
+  return sizeof(T) * (size_t)(2 * NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB);
 }
 
 template <typename T, bool COLTYPE, bool BACKWARD, bool UNIT>
@@ -536,14 +597,16 @@ int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int6
   constexpr int NB = Geo<T>::NB, V = Geo<T>::V, WPE = Words<T>::N;
   *handled = false;
   if (!knob(kKnobTrsvFront)) return B2_STATUS_OK;
+  // Column-type views (op(A)'s rows strided in memory) load their sub-blocks from 16 memory rows
+  // per request; the block-row kernel is faster there.
+  if (coltype && knob(kKnobTrsvFront) < 2) return B2_STATUS_OK;
   if (!aligned_to(a, 16) || lda % V != 0) return B2_STATUS_OK;
   const int64_t nb64 = (n + NB - 1) / NB;
   if (nb64 > 0x3fffffff) return B2_STATUS_OK;
   const int nb = (int)nb64;
   const int grid = nb < sm_count() ? nb : sm_count();
   const size_t xbuf_words = (size_t)nb * NB * WPE;
-  const size_t dump_words = (size_t)grid * 2 * NB * WPE;
-  if ((xbuf_words + dump_words) * 8 > l.scratch_bytes) return B2_STATUS_OK;
+  if (xbuf_words * 8 > l.scratch_bytes) return B2_STATUS_OK;
   FrontArgs<T> args = {};
   args.a = a;
   args.lda = lda;
@@ -551,7 +614,6 @@ int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int6
   args.x = xbase;
   args.incx = incx;
   args.xbuf = reinterpret_cast<unsigned long long*>(l.scratch);
-  args.dump = args.xbuf + xbuf_words;
   args.ctl = l.ctl;
   args.nb = nb;
   {  // keep the prefetched-but-unused tiles of all blocks within a fraction of L2
@@ -563,6 +625,9 @@ int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int6
   args.wait_limit = l.wait_limit;
   args.device_status = l.device_status;
   args.debug_skip = (int)knob(kKnobTrsvDebugSkip);
+#ifdef B2_TRSV_TRACE
+  args.trace = reinterpret_cast<unsigned long long*>(l.scratch + l.scratch_bytes - ((size_t)16 << 20));
+#endif
   *handled = true;
   if (coltype)
     return backward ? launch_diag<T, true, true>(l, args, grid, unit) : launch_diag<T, true, false>(l, args, grid, unit);
