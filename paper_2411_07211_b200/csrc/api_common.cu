@@ -14,6 +14,7 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobTriWide         */ 0,
     /* kKnobTrsvPrefetchBytes */ 48 << 20,
     /* kKnobTrsvFront       */ 1,
+    /* kKnobTrsvCluster     */ 1,
 };
 
 unsigned long long g_launch_count = 0;

@@ -80,8 +80,42 @@ __device__ __forceinline__ void bar_sync(int id, int count) {
   __syncwarp();
   asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
+// Polling load through a generic address: the words live in global memory (another cluster's
+// row) or in this block's shared memory (a row of the same cluster, written by its block).
 __device__ __forceinline__ void ld_word2(const unsigned long long* p, unsigned long long& a, unsigned long long& b) {
-  asm volatile("ld.relaxed.gpu.global.v2.u64 {%0,%1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+  asm volatile("ld.relaxed.gpu.v2.u64 {%0,%1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
+// Thread-block cluster pieces: rank, cluster-wide barrier, address of a peer's shared memory,
+// (predicated) stores into it.
+__device__ __forceinline__ unsigned cluster_rank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ unsigned map_remote(const void* local_smem, unsigned rank) {
+  unsigned r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"((unsigned)__cvta_generic_to_shared(local_smem)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_remote_u32(unsigned raddr, unsigned v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(raddr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_remote_if(bool pred, unsigned raddr, unsigned long long v) {
+  asm volatile("{ .reg .pred q; setp.ne.u32 q, %0, 0; @q st.shared::cluster.u64 [%1], %2; }" ::"r"((unsigned)pred),
+               "r"(raddr), "l"(v)
+               : "memory");
+}
+__device__ __forceinline__ void publish_remote_if(bool pred, unsigned raddr, float v, unsigned tag) {
+  st_remote_if(pred, raddr, ((unsigned long long)tag << 32) | __float_as_uint(v));
+}
+__device__ __forceinline__ void publish_remote_if(bool pred, unsigned raddr, double v, unsigned tag) {
+  const unsigned long long b = (unsigned long long)__double_as_longlong(v);
+  st_remote_if(pred, raddr, ((unsigned long long)tag << 32) | (b & 0xffffffffull));
+  st_remote_if(pred, raddr + 8, ((unsigned long long)tag << 32) | (b >> 32));
 }
 // Stores under a predicate instead of a branch: the instructions are fetched on every trip of
 // the tile loop and take effect on the last one only.
@@ -124,7 +158,6 @@ __device__ __forceinline__ double decode(const unsigned long long* w, double) {
 // Per-thread state of the bounded waits.
 struct Waiter {
   unsigned long long budget;
-  unsigned tag;
   unsigned* abort_word;  // control block: raised by the first wait that runs out
   int* device_status;
   bool dead;             // this thread stopped waiting (its budget ran out, or the abort word is up)
@@ -137,7 +170,7 @@ struct Waiter {
   // w holds a first attempt at the four words ptr[0..3] (16-byte aligned); polls until the
   // words with their bit in `need` set carry this call's tag.
   __device__ __forceinline__ void finish(unsigned long long (&w)[4], const unsigned long long* ptr, unsigned need,
-                                         unsigned sleep_ns) {
+                                         unsigned tag, unsigned sleep_ns) {
     if (need == 0u) return;
     for (;;) {
       bool ok = true;
@@ -188,7 +221,11 @@ __device__ __forceinline__ void st4(double* p, double a, double b, double c, dou
 
 // ---------------------------------------------------------------------------------------
 // COLTYPE: op(A)'s rows are columns of the stored row-major view.  BACKWARD: solve bottom-up.
-template <typename T, bool COLTYPE, bool BACKWARD, bool UNIT>
+// CS: blocks per cluster (1 = no cluster).  With CS = 8 a cluster takes eight consecutive block
+// rows; a solved block is also written straight into the shared memory of the blocks that
+// hold the later rows of the cluster, so seven hand-overs out of eight skip the trip through
+// L2 and the polling of global memory.
+template <typename T, bool COLTYPE, bool BACKWARD, bool UNIT, int CS>
 __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p) {
   constexpr int NB = Geo<T>::NB, V = Geo<T>::V, WPE = Words<T>::N;
   constexpr int RS = NB / 16;  // sub-block edge: 8 (float) / 4 (double)
@@ -206,6 +243,8 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
   T* xs = Wt + NB * SP;                         // [2][NB] x values of the current / next tile
   T* rbuf = xs + 2 * NB;                        // r = b - sum, the vector of the final trip
   T* bvec = rbuf + NB;
+  // x of the earlier rows of this cluster: [CS][NB * WPE] words {payload, row + 1}, written by their blocks
+  unsigned long long* xrecv = reinterpret_cast<unsigned long long*>(bvec + NB);
   __shared__ unsigned s_ticket[2];
 #ifdef B2_TRSV_TRACE
   __shared__ unsigned long long s_trace[16];
@@ -219,23 +258,35 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
 
   Waiter wt;
   wt.budget = p.wait_limit ? p.wait_limit : (1ull << 22);
-  wt.tag = p.tag;
   wt.abort_word = p.ctl + kCtlTrsvAbort;
   wt.device_status = p.device_status;
   wt.dead = false;
   int parity = 0;
+  const unsigned rank = CS > 1 ? cluster_rank() : 0u;
+  if (CS > 1) {
+    for (int i = ct; i < CS * NB * WPE; i += kT) xrecv[i] = 0ull;  // no stale word may look like a row of this call
+    cluster_sync_all();
+  }
 
   for (;;) {
-    if (ct == 0) {
+    // one ticket per cluster = CS consecutive block rows in solve order
+    if (rank == 0u && ct == 0) {
       unsigned kk = 0xffffffffu;
       if (!wt.dead && ld_flag(wt.abort_word) == 0u) kk = atomicAdd(p.ctl + kCtlTrsvTicket, 1u);
-      s_ticket[parity] = kk;
+      if (CS > 1) {
+        for (unsigned r = 0; r < (unsigned)CS; ++r) st_remote_u32(map_remote(&s_ticket[parity], r), kk);
+      } else {
+        s_ticket[parity] = kk;
+      }
     }
-    bar_sync(kBar, kT);
-    const unsigned kk = s_ticket[parity];
+    if (CS > 1) cluster_sync_all();
+    else bar_sync(kBar, kT);
+    const unsigned long long kk = (unsigned long long)s_ticket[parity] * CS + rank;
     parity ^= 1;
-    if (kk >= (unsigned)p.nb) break;
+    if (kk - rank >= (unsigned long long)p.nb) break;  // the whole cluster leaves together
+    if (kk >= (unsigned long long)p.nb) continue;     // this group has fewer than CS rows
     const int k = (int)kk;  // position in the solve order = number of source tiles
+    const int g0 = k - (int)rank;  // first row of this cluster's group
     B2_CTRACE(ct == 0, 0);
     const int I = BACKWARD ? p.nb - 1 - k : k;
     const int64_t r0 = (int64_t)I * NB;
@@ -473,13 +524,14 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
 
     B2_CTRACE(ct == 0, 1);
     // --- along the block row; trip `k` (the last) applies the inverse
-    T cur[E], nxt[E];
-    load_tile(cur, 0);
+    // two register sets take turns: while one is multiplied, the other receives the next tile
+    T tile_a[E], tile_b[E];
+    load_tile(tile_a, 0);
     const T bi = bvec[ti];
     T racc = T(0);
     // warp 0 fetches the x values of a tile: 4 tagged words per lane, first attempt one trip ahead
     unsigned long long xw[4] = {0, 0, 0, 0};
-    unsigned xneed = 0;
+    unsigned xneed = 0, xtag = p.tag;
     const unsigned long long* xptr = p.xbuf;
     auto x_issue = [&](int s) {
       const int64_t xi = (int64_t)blk(s) * NB + V * lane;
@@ -487,7 +539,9 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
 #pragma unroll
       for (int e = 0; e < V; ++e)
         if (xi + e < p.n) xneed |= ((1u << WPE) - 1u) << (e * WPE);
-      xptr = p.xbuf + xi * WPE;
+      const bool local = CS > 1 && s >= g0;  // a row of this cluster: its block writes into xrecv
+      xptr = local ? xrecv + ((s - g0) * NB + V * lane) * WPE : p.xbuf + xi * WPE;
+      xtag = local ? (unsigned)s + 1u : p.tag;
       if (xneed) {
         ld_word2(xptr, xw[0], xw[1]);
         ld_word2(xptr + 2, xw[2], xw[3]);
@@ -495,10 +549,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     };
     if (warp == 0 && k > 0) x_issue(0);
 
-    int ntrips = k + 1;
-    asm volatile("" : "+r"(ntrips));  // one loop, not a peeled copy of its last trip
-#pragma unroll 1
-    for (int it = 0; it < ntrips; ++it) {
+    auto trip = [&](T (&cur)[E], T (&nxt)[E], int it) {
       const bool last = it == k;
       T* xbuf_s = xs + (it & 1) * NB;
       // first of all, off the critical path: the next tile (or the inverse) into the second
@@ -508,7 +559,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       if (warp == 0 && !last) {
         const int dist = k - it;  // rows between this block and the producer of the tile's x
         B2_CTRACE(ct == 0 && it == k - 1, 2);
-        wt.finish(xw, xptr, xneed, dist > 2 ? (unsigned)min((dist - 2) * 200, 2000) : 0u);
+        wt.finish(xw, xptr, xneed, xtag, dist > 2 ? (unsigned)min((dist - 2) * 200, 2000) : 0u);
         B2_CTRACE(ct == 0 && it == k - 1, 3);
         P xv;
 #pragma unroll
@@ -539,19 +590,33 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       if (owner && !last) rbuf[ti] = bi - racc;
       {  // publishing stores: fetched on every trip, performed on the last
         const bool real = last && owner && row_ok && !wt.dead && k != p.debug_skip;
+        if (CS > 1) {  // first of all to the blocks that hold the later rows of this cluster
+#pragma unroll
+          for (int rr = 1; rr < CS; ++rr) {
+            const unsigned target = min(rank + (unsigned)rr, (unsigned)CS - 1u);
+            publish_remote_if(real && rank + (unsigned)rr < (unsigned)CS, map_remote(xrecv + ((int)rank * NB + mi) * WPE, target),
+                              s, (unsigned)k + 1u);
+          }
+        }
         publish_if(real, p.xbuf + (r0 + mi) * WPE, s, p.tag);
         st_val_if(real, p.x + (r0 + mi) * p.incx, s);
       }
       B2_CTRACE(ct == 0 && last, 4);
       if (warp == 0 && it + 1 < k) x_issue(it + 1);  // first attempt at the x words of the next tile
-#pragma unroll
-      for (int e = 0; e < E; ++e) cur[e] = nxt[e];
+    };
+    int ntrips = k + 1;
+    asm volatile("" : "+r"(ntrips));  // loops of two trips, not peeled copies of the last ones
+#pragma unroll 1
+    for (int it = 0; it < ntrips; it += 2) {
+      trip(tile_a, tile_b, it);
+      if (it + 1 < ntrips) trip(tile_b, tile_a, it + 1);
     }
     bar_sync(kBar, kT);  // S, bvec, rbuf, xs are reused by the next block row
 #ifdef B2_TRSV_TRACE
     if (ct < 16) p.trace[k * 16 + ct] = s_trace[ct];
 #endif
   }
+  if (CS > 1) cluster_sync_all();  // no block leaves while a peer may still write into its shared memory
   // The last block out leaves the control block clean (not after an abort: the caller resets).
   if (ct == 0 && ld_flag(p.ctl + kCtlTrsvAbort) == 0u) {
     __threadfence();
@@ -564,28 +629,64 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
 }
 
 template <typename T>
-constexpr size_t front_smem_bytes() {
+constexpr size_t front_smem_bytes(int cs) {
   constexpr int NB = Geo<T>::NB;
   constexpr int SP = NB + 16 / (int)sizeof(T);
-  return sizeof(T) * (size_t)(2 * NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB);
+  return sizeof(T) * (size_t)(2 * NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB) +
+         (cs > 1 ? (size_t)cs * NB * Words<T>::N * 8 : 0);
 }
 
+constexpr int kCluster = 8;
+
+// Launches the kernel; with clusters when the device can hold at least one (the grid is then a
+// whole number of clusters, no more than can be resident), else block by block.
 template <typename T, bool COLTYPE, bool BACKWARD, bool UNIT>
-static int launch_one(const Launch& l, const FrontArgs<T>& args, int grid) {
-  constexpr size_t smem = front_smem_bytes<T>();
-  auto kern = trsv_front_kernel<T, COLTYPE, BACKWARD, UNIT>;
+static int launch_one(const Launch& l, const FrontArgs<T>& args, int nb, bool want_cluster) {
+  if (want_cluster) {
+    constexpr size_t smem = front_smem_bytes<T>(kCluster);
+    auto kern = trsv_front_kernel<T, COLTYPE, BACKWARD, UNIT, kCluster>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess) {
+      cudaLaunchConfig_t cfg = {};
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = kCluster;
+      at[0].val.clusterDim.y = 1;
+      at[0].val.clusterDim.z = 1;
+      cfg.gridDim = dim3(kCluster);
+      cfg.blockDim = dim3(kT);
+      cfg.dynamicSmemBytes = smem;
+      cfg.stream = l.stream;
+      cfg.attrs = at;
+      cfg.numAttrs = 1;
+      int max_clusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg) == cudaSuccess && max_clusters > 0) {
+        const int groups = (nb + kCluster - 1) / kCluster;
+        const int clusters = groups < max_clusters ? groups : max_clusters;
+        cfg.gridDim = dim3(clusters * kCluster);
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, args);
+        ++g_launch_count;
+        if (e == cudaSuccess) return B2_STATUS_OK;
+        (void)cudaGetLastError();
+        return B2_STATUS_LAUNCH_FAILED;
+      }
+    }
+    (void)cudaGetLastError();
+  }
+  constexpr size_t smem = front_smem_bytes<T>(1);
+  auto kern = trsv_front_kernel<T, COLTYPE, BACKWARD, UNIT, 1>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     (void)cudaGetLastError();
     return B2_STATUS_LAUNCH_FAILED;
   }
+  const int grid = nb < sm_count() ? nb : sm_count();
   kern<<<grid, kT, smem, l.stream>>>(args);
   return check_launch();
 }
 
 template <typename T, bool COLTYPE, bool BACKWARD>
-static int launch_diag(const Launch& l, const FrontArgs<T>& args, int grid, bool unit) {
-  return unit ? launch_one<T, COLTYPE, BACKWARD, true>(l, args, grid)
-              : launch_one<T, COLTYPE, BACKWARD, false>(l, args, grid);
+static int launch_diag(const Launch& l, const FrontArgs<T>& args, int nb, bool want_cluster, bool unit) {
+  return unit ? launch_one<T, COLTYPE, BACKWARD, true>(l, args, nb, want_cluster)
+              : launch_one<T, COLTYPE, BACKWARD, false>(l, args, nb, want_cluster);
 }
 
 }  // namespace tf
@@ -629,9 +730,14 @@ int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int6
   args.trace = reinterpret_cast<unsigned long long*>(l.scratch + l.scratch_bytes - ((size_t)16 << 20));
 #endif
   *handled = true;
+  // (measured: clusters pay for float; for double, with twice the words per value to push to
+  // seven peers, they do not)
+  const bool want_cluster = nb >= 2 && (knob(kKnobTrsvCluster) >= 2 || (knob(kKnobTrsvCluster) == 1 && sizeof(T) == 4));
   if (coltype)
-    return backward ? launch_diag<T, true, true>(l, args, grid, unit) : launch_diag<T, true, false>(l, args, grid, unit);
-  return backward ? launch_diag<T, false, true>(l, args, grid, unit) : launch_diag<T, false, false>(l, args, grid, unit);
+    return backward ? launch_diag<T, true, true>(l, args, nb, want_cluster, unit)
+                    : launch_diag<T, true, false>(l, args, nb, want_cluster, unit);
+  return backward ? launch_diag<T, false, true>(l, args, nb, want_cluster, unit)
+                  : launch_diag<T, false, false>(l, args, nb, want_cluster, unit);
 }
 
 template int trsv_front_try<float>(const Launch&, bool, bool, bool, int64_t, const float*, int64_t, float*, int64_t,
