@@ -235,12 +235,14 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
   constexpr int SP = NB + 16 / (int)sizeof(T);  // row pitch of S (rows start 16-byte aligned)
   constexpr bool CANON_LOWER = (COLTYPE == BACKWARD);  // stored triangle in the row-major view
   using P = Pack<T, V>;
+  constexpr bool PM = CS == 1;  // premultiply the last tile (see below)
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* S = reinterpret_cast<T*>(smem_raw);       // diagonal block, then its inverse (symmetric storage)
   T* Tm = S + NB * SP;                          // products in flight during the inversion
   T* Wt = Tm + (NB / 2) * (NB / 2 + 4);         // the finished inverse in the tile loader's layout
-  T* xs = Wt + NB * SP;                         // [2][NB] x values of the current / next tile
+  T* Ms = Wt + NB * SP;                         // inv(D_k) * A_{k,k-1} in the same layout (the tile of the last trip)
+  T* xs = Ms + (PM ? NB * SP : 0);              // [2][NB] x values of the current / next tile
   T* rbuf = xs + 2 * NB;                        // r = b - sum, the vector of the final trip
   T* bvec = rbuf + NB;
   // x of the earlier rows of this cluster: [CS][NB * WPE] words {payload, row + 1}, written by their blocks
@@ -299,14 +301,19 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     // tile s of this block row -> registers: m[a * RS + b] = op(A)(row sub_i(a), column sub_j(b)).
     // A thread's RS rows / columns are two chunks of V (one 16-byte pack), NB/2 apart: the packs
     // that the lanes of a warp load together then tile whole 32-byte sectors.
-    // "Tile" k is the inverse of the diagonal block, laid out in shared memory (Wt) so that the
-    // very same loads fetch it: the addresses are generic.
-    auto load_tile = [&](T (&m)[E], int s) {
-      const bool inv = s == k;
+    // The tiles of the last two trips are inv(D_k) and inv(D_k) A_{k,k-1}, laid out in shared
+    // memory (Wt, Ms) so that the very same loads fetch them: the addresses are generic.
+    // PM (premultiply): the last tile is replaced by inv(D_k) A_{k,k-1}, so that one product instead
+    // of two stands between x_{k-1} and x_k -- at the price of two trips between x_{k-2} and
+    // x_{k-1}.  It pays where the hand-over itself is slow (through L2), not inside a cluster.
+    const int nm = (PM && k > 0) ? 1 : 0;
+    const int yt = k - nm;  // the trip that applies inv(D_k) to b - sum
+    auto load_tile = [&](T (&m)[E], int s, bool raw) {
+      const bool inv = !raw && s >= yt;  // trip yt reads Wt, trip k > 0 reads Ms; `raw`: the matrix tile itself
       const int64_t c0 = inv ? 0 : (int64_t)blk(s) * NB;
       const int nbJ = inv ? NB : (int)min((int64_t)NB, p.n - c0);
       if (inv || (nbI == NB && nbJ == NB)) {
-        const T* base = inv ? Wt : p.a;
+        const T* base = inv ? (s == yt ? Wt : Ms) : p.a;
         const int64_t ld = inv ? SP : p.lda, rr0 = inv ? 0 : r0;
         if (!COLTYPE) {
 #pragma unroll
@@ -401,6 +408,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     }
     for (int s = ct; s < NB; s += kT)
       if (s >= nbI) S[s * SP + s] = T(1);
+    prefetch_tile(k - 1);
     for (int s = 0; s < p.pf_dist; ++s) prefetch_tile(s);
     bar_sync(kBar, kT);
 
@@ -520,16 +528,74 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       const int j = COLTYPE ? rho : gam;
       Wt[rho * SP + gam] = j <= i ? S[i * SP + j] : T(0);
     }
+    // --- Ms = inv(D_k) * A_{k,k-1}: with it, x_k = inv(D_k) (b - earlier tiles) - Ms x_{k-1}, and only
+    // ONE tile-times-vector product stands between the arrival of x_{k-1} and x_k.
+    if (nm) {
+      {  // the tile, rows in solve order, through registers into Ms
+        T t1[E];
+        load_tile(t1, k - 1, true);
+#pragma unroll
+        for (int a = 0; a < RS; ++a)
+#pragma unroll
+          for (int hb = 0; hb < RS / V; ++hb) {
+            P pk;
+#pragma unroll
+            for (int e = 0; e < V; ++e) pk.v[e] = t1[a * RS + hb * V + e];
+            *reinterpret_cast<P*>(Ms + ((a / V) * H + V * rg + (a % V)) * SP + hb * H + V * cg) = pk;
+          }
+      }
+      bar_sync(kBar, kT);
+      constexpr int JW = NB * NB / (4 * kT);  // columns per thread: 16 (float) / 4 (double), 4 rows
+      constexpr int NJQ = NB / JW;            // threads along a row; a thread's chunks of 4 columns are 4 * NJQ apart
+      const int i0 = (ct / NJQ) * 4, j0 = (ct % NJQ) * 4;
+      T acc[4][JW];
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+        for (int jj = 0; jj < JW; ++jj) acc[ii][jj] = T(0);
+#pragma unroll 2
+      for (int l = 0; l < i0 + 4; ++l) {  // inv(D_k) is zero above its diagonal
+        T wv[4];
+        ld4(S + l * SP + i0, wv);  // column l of the inverse, through the mirrored half of S
+#pragma unroll
+        for (int ii = 0; ii < 4; ++ii)
+          if (i0 + ii < l) wv[ii] = T(0);
+#pragma unroll
+        for (int u = 0; u < JW / 4; ++u) {
+          T tv[4];
+          ld4(Ms + l * SP + j0 + u * 4 * NJQ, tv);
+#pragma unroll
+          for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[ii][u * 4 + e] = wv[ii] * tv[e] + acc[ii][u * 4 + e];
+        }
+      }
+      bar_sync(kBar, kT);  // everybody has read the tile: overwrite it with the product, in the loader's layout
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii) {
+        const int i = i0 + ii, mrow = BACKWARD ? NB - 1 - i : i;
+        if (!COLTYPE) {
+#pragma unroll
+          for (int u = 0; u < JW / 4; ++u)
+            st4(Ms + mrow * SP + j0 + u * 4 * NJQ, acc[ii][u * 4], acc[ii][u * 4 + 1], acc[ii][u * 4 + 2], acc[ii][u * 4 + 3]);
+        } else {
+#pragma unroll
+          for (int jj = 0; jj < JW; ++jj) Ms[(j0 + (jj / 4) * 4 * NJQ + jj % 4) * SP + mrow] = acc[ii][jj];
+        }
+      }
+    }
     bar_sync(kBar, kT);
 
     B2_CTRACE(ct == 0, 1);
-    // --- along the block row; trip `k` (the last) applies the inverse
+    // --- along the block row.  Trips 0 .. k-2 multiply the tiles A_ks by x_s and add up; trip
+    // yt = k-1 multiplies inv(D_k) by r = b - sum (y); trip k multiplies Ms by x_{k-1}: x_k = y - that.
+    // (Row 0 has the single trip yt = 0 and x_0 = y.)
     // two register sets take turns: while one is multiplied, the other receives the next tile
     T tile_a[E], tile_b[E];
-    load_tile(tile_a, 0);
+    load_tile(tile_a, 0, false);
     const T bi = bvec[ti];
-    T racc = T(0);
-    // warp 0 fetches the x values of a tile: 4 tagged words per lane, first attempt one trip ahead
+    T racc = T(0), yreg = T(0);
+    // warp 0 fetches the x values a trip needs: 4 tagged words per lane, first attempt one trip ahead
     unsigned long long xw[4] = {0, 0, 0, 0};
     unsigned xneed = 0, xtag = p.tag;
     const unsigned long long* xptr = p.xbuf;
@@ -547,29 +613,31 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
         ld_word2(xptr + 2, xw[2], xw[3]);
       }
     };
-    if (warp == 0 && k > 0) x_issue(0);
+    if (warp == 0 && k > 0) x_issue(yt > 0 ? 0 : k - 1);  // (yt == 0 < k only with PM: the M trip's x)
 
     auto trip = [&](T (&cur)[E], T (&nxt)[E], int it) {
-      const bool last = it == k;
+      const bool is_y = it == yt;
+      const bool is_m = nm && it == k;
+      const bool crit = it == k;  // the trip that ends with x_k
+      const int srow = is_m ? k - 1 : it;      // the block whose x this trip multiplies (none on trip yt)
       T* xbuf_s = xs + (it & 1) * NB;
-      // first of all, off the critical path: the next tile (or the inverse) into the second
-      // register set and a tile further ahead towards L2 -- in flight while this trip waits
-      if (!last) load_tile(nxt, it + 1);
+      // first of all, off the critical path: the next tile into the other register set and a
+      // tile further ahead towards L2 -- in flight while this trip waits
+      if (it < k) load_tile(nxt, it + 1, false);
       prefetch_tile(it + 1 + p.pf_dist);
-      if (warp == 0 && !last) {
-        const int dist = k - it;  // rows between this block and the producer of the tile's x
-        B2_CTRACE(ct == 0 && it == k - 1, 2);
+      if (warp == 0 && !is_y) {
+        const int dist = k - srow;  // rows between this block and the producer of the x
+        B2_CTRACE(ct == 0 && srow == k - 1, 2);
         wt.finish(xw, xptr, xneed, xtag, dist > 2 ? (unsigned)min((dist - 2) * 200, 2000) : 0u);
-        B2_CTRACE(ct == 0 && it == k - 1, 3);
+        B2_CTRACE(ct == 0 && srow == k - 1, 3);
         P xv;
 #pragma unroll
         for (int e = 0; e < V; ++e) xv.v[e] = ((xneed >> (e * WPE)) & 1u) ? decode(xw + e * WPE, T(0)) : T(0);
         *reinterpret_cast<P*>(xbuf_s + V * lane) = xv;
       }
       bar_sync(kBar, kT);
-      B2_CTRACE(ct == 0 && it == k - 1, 8);
-      B2_CTRACE(ct == 0 && last, 9);
-      const T* vec = last ? rbuf : xbuf_s;
+      B2_CTRACE(ct == 0 && srow == k - 1 && !is_y, 8);
+      const T* vec = is_y ? rbuf : xbuf_s;
       T xv[RS], part[RS];
 #pragma unroll
       for (int hb = 0; hb < RS / V; ++hb) {
@@ -584,25 +652,31 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
         for (int bcol = 0; bcol < RS; ++bcol) part[a] = cur[a * RS + bcol] * xv[bcol] + part[a];
       }
       const T s = multi_group_sum<16, RS>(part, lane);
-      B2_CTRACE(ct == 0 && it == k - 1, 7);
-      B2_CTRACE(ct == 0 && last, 10);
-      if (!last) racc += s;
-      if (owner && !last) rbuf[ti] = bi - racc;
+      B2_CTRACE(ct == 0 && srow == k - 1 && !is_y, 7);
+      const T out = is_m ? yreg - s : s;
+      if (is_y) yreg = s;
+      if (it < yt) racc += s;
+      if (owner && it < yt) rbuf[ti] = bi - racc;
       {  // publishing stores: fetched on every trip, performed on the last
-        const bool real = last && owner && row_ok && !wt.dead && k != p.debug_skip;
-        if (CS > 1) {  // first of all to the blocks that hold the later rows of this cluster
+        const bool real = crit && owner && row_ok && !wt.dead && k != p.debug_skip;
+        if (CS > 1) {  // first of all to the blocks that hold the later rows of this cluster: they
+                       // are one, two, ... steps away from needing it, and a trip takes most of a step
 #pragma unroll
           for (int rr = 1; rr < CS; ++rr) {
             const unsigned target = min(rank + (unsigned)rr, (unsigned)CS - 1u);
             publish_remote_if(real && rank + (unsigned)rr < (unsigned)CS, map_remote(xrecv + ((int)rank * NB + mi) * WPE, target),
-                              s, (unsigned)k + 1u);
+                              out, (unsigned)k + 1u);
           }
         }
-        publish_if(real, p.xbuf + (r0 + mi) * WPE, s, p.tag);
-        st_val_if(real, p.x + (r0 + mi) * p.incx, s);
+        publish_if(real, p.xbuf + (r0 + mi) * WPE, out, p.tag);
+        st_val_if(real, p.x + (r0 + mi) * p.incx, out);
       }
-      B2_CTRACE(ct == 0 && last, 4);
-      if (warp == 0 && it + 1 < k) x_issue(it + 1);  // first attempt at the x words of the next tile
+      B2_CTRACE(ct == 0 && crit, 4);
+      // first attempt at the x words of the next trip that needs some
+      if (warp == 0) {
+        if (it + 1 < yt) x_issue(it + 1);
+        else if (it + 1 == yt && nm) x_issue(k - 1);
+      }
     };
     int ntrips = k + 1;
     asm volatile("" : "+r"(ntrips));  // loops of two trips, not peeled copies of the last ones
@@ -632,7 +706,7 @@ template <typename T>
 constexpr size_t front_smem_bytes(int cs) {
   constexpr int NB = Geo<T>::NB;
   constexpr int SP = NB + 16 / (int)sizeof(T);
-  return sizeof(T) * (size_t)(2 * NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB) +
+  return sizeof(T) * (size_t)((cs > 1 ? 2 : 3) * NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB) +
          (cs > 1 ? (size_t)cs * NB * Words<T>::N * 8 : 0);
 }
 
