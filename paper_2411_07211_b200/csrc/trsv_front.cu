@@ -240,8 +240,8 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* S = reinterpret_cast<T*>(smem_raw);       // diagonal block, then its inverse (symmetric storage)
   T* Tm = S + NB * SP;                          // products in flight during the inversion
-  T* Wt = Tm + (NB / 2) * (NB / 2 + 4);         // the finished inverse in the tile loader's layout
-  T* Ms = Wt + NB * SP;                         // inv(D_k) * A_{k,k-1} in the same layout (the tile of the last trip)
+  T* Wt = S;                                    // ... and finally the inverse in the tile loader's layout
+  T* Ms = Tm + (NB / 2) * (NB / 2 + 4);         // inv(D_k) * A_{k,k-1} in the same layout (the tile of the last trip)
   T* xs = Ms + (PM ? NB * SP : 0);              // [2][NB] x values of the current / next tile
   T* rbuf = xs + 2 * NB;                        // r = b - sum, the vector of the final trip
   T* bvec = rbuf + NB;
@@ -521,13 +521,6 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       }
       bar_sync(kBar, kT);
     }
-    // --- the inverse (zero above its diagonal) -> Wt, indexed the way load_tile reads a tile
-    for (int idx = ct; idx < NB * NB; idx += kT) {
-      const int rho = idx / NB, gam = idx % NB;
-      const int i = COLTYPE ? (BACKWARD ? NB - 1 - gam : gam) : (BACKWARD ? NB - 1 - rho : rho);
-      const int j = COLTYPE ? rho : gam;
-      Wt[rho * SP + gam] = j <= i ? S[i * SP + j] : T(0);
-    }
     // --- Ms = inv(D_k) * A_{k,k-1}: with it, x_k = inv(D_k) (b - earlier tiles) - Ms x_{k-1}, and only
     // ONE tile-times-vector product stands between the arrival of x_{k-1} and x_k.
     if (nm) {
@@ -582,6 +575,29 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
 #pragma unroll
           for (int jj = 0; jj < JW; ++jj) Ms[(j0 + (jj / 4) * 4 * NJQ + jj % 4) * SP + mrow] = acc[ii][jj];
         }
+      }
+    }
+    bar_sync(kBar, kT);
+
+    // --- the inverse, in place, into the layout in which load_tile reads a tile: zero above the
+    // diagonal, rows (row-type views) or columns (column-type views) reversed for a bottom-up solve
+    for (int idx = ct; idx < NB * NB / 2; idx += kT) {
+      if (!BACKWARD) {  // only the masking: two elements per thread and step
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int e2 = idx + half * (NB * NB / 2), rho = e2 / NB, gam = e2 % NB;
+          if (COLTYPE ? rho > gam : gam > rho) S[rho * SP + gam] = T(0);
+        }
+      } else if (!COLTYPE) {  // swap row rho with row NB-1-rho
+        const int rho = idx / NB, gam = idx % NB, rho2 = NB - 1 - rho;
+        const T va = S[rho * SP + gam], vb = S[rho2 * SP + gam];
+        S[rho * SP + gam] = gam <= rho2 ? vb : T(0);
+        S[rho2 * SP + gam] = gam <= rho ? va : T(0);
+      } else {  // swap column gam with column NB-1-gam
+        const int rho = idx / (NB / 2), gam = idx % (NB / 2), gam2 = NB - 1 - gam;
+        const T va = S[rho * SP + gam], vb = S[rho * SP + gam2];
+        S[rho * SP + gam] = rho <= gam2 ? vb : T(0);
+        S[rho * SP + gam2] = rho <= gam ? va : T(0);
       }
     }
     bar_sync(kBar, kT);
@@ -706,7 +722,7 @@ template <typename T>
 constexpr size_t front_smem_bytes(int cs) {
   constexpr int NB = Geo<T>::NB;
   constexpr int SP = NB + 16 / (int)sizeof(T);
-  return sizeof(T) * (size_t)((cs > 1 ? 2 : 3) * NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB) +
+  return sizeof(T) * (size_t)((cs > 1 ? 1 : 2) * NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB) +
          (cs > 1 ? (size_t)cs * NB * Words<T>::N * 8 : 0);
 }
 
