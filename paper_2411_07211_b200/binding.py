@@ -28,7 +28,7 @@ STATUS_TOO_LARGE = 6
 KNOB_L1_BLOCKS_PER_SM, KNOB_GEMV_N_TILE_BYTES, KNOB_GEMV_T_ROWS, KNOB_TRI_ROWS = 0, 1, 2, 3
 KNOB_GER_ROWS, KNOB_USE_PDL, KNOB_TRSV_DEBUG_SKIP, KNOB_TRI_WIDE = 4, 5, 6, 7
 KNOB_TRSV_PREFETCH_BYTES = 8
-KNOB_TRSV_FRONT = 9
+KNOB_TRSV_FRONT, KNOB_TRSV_CLUSTER = 9, 10
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libb2blas.so")
 

@@ -195,8 +195,8 @@ enum Knob {
   kKnobTrsvDebugSkip = 6,  // test hook: solve-order block that never publishes (-1 = none)
   kKnobTriWide = 7,
   kKnobTrsvPrefetchBytes = 8,  // total L2 bytes trsv blocks may prefetch ahead of the front
-  kKnobTrsvCluster = 10,       // sub-block trsv: 1 = clusters of 8 consecutive block rows with hand-over through shared memory
-  kKnobTrsvFront = 9,          // 1: sub-block trsv kernel where its preconditions hold; 0: general block-row kernel
+  kKnobTrsvFront = 9,          // 0: block-row trsv kernel only; 1: sub-block kernel for row-type views; 2: for all views
+  kKnobTrsvCluster = 10,       // sub-block trsv in clusters of 8 block rows: 0 never, 1 float only, 2 always
   kKnobCount = 16
 };
 int64_t knob(int id);

@@ -7,11 +7,13 @@
 // rows in solve order.  A block
 //   1. inverts its diagonal block D_k in shared memory long before the front arrives
 //      (recursive doubling on 4x4 register tiles; the matrix is kept in symmetric storage so
-//      that both operand orientations are contiguous) and keeps inv(D_k) in registers,
+//      that both operand orientations are contiguous) and leaves inv(D_k) there in the
+//      layout of a matrix tile,
 //   2. walks along its block row: tile A_ks sits in registers, distributed over a 16 x 16
 //      thread grid (an RS x RS sub-block per thread), so a tile-times-vector product needs RS
 //      vector elements per thread from shared memory and one RS-value reduction over the 16
-//      lanes of a row group -- a few hundred cycles from "x_s is here" to "row sums updated",
+//      lanes of a row group -- a few hundred cycles from "x_s is here" to "row sums updated";
+//      two register sets take turns, one multiplied while the other receives the next tile,
 //   3. treats inv(D_k) as one more tile whose vector is r = b - sum: the last trip through the
 //      SAME loop body produces x_k.  That matters: a stretch of code that a block executes
 //      once, after tens of microseconds of doing something else, costs microseconds of

@@ -206,6 +206,34 @@ def test_trsv_bounded_wait_reports_timeout(b2):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("front,cluster", [(0, 0), (2, 0), (2, 2)])
+def test_trsv_every_kernel_choice(b2, ctx, dtype, front, cluster):
+    """trsv has three code paths (block-row kernel; sub-block kernel block by block, which
+    premultiplies the last tile; sub-block kernel in clusters).  The defaults pick one per
+    precision and view; here each is forced for every view, on sizes with a ragged last block
+    and more block rows than one cluster holds."""
+    old = b2.get_tuning(b2.KNOB_TRSV_FRONT), b2.get_tuning(b2.KNOB_TRSV_CLUSTER)
+    b2.set_tuning(b2.KNOB_TRSV_FRONT, front)
+    b2.set_tuning(b2.KNOB_TRSV_CLUSTER, cluster)
+    try:
+        tol = TOL[np.dtype(dtype)]
+        for n in (130, 1100, 2052):
+            for uplo, trans, diag in itertools.product(UPLOS, TRANSES, DIAGS):
+                a = tri_buf(21, n, n, dtype, orc.ROW_MAJOR, uplo, diag)
+                hx = synth.vector_np(9, n, n, dtype)
+                ga, gx = Guarded(a), Guarded(hx)
+                b2.trsv(ctx, orc.ROW_MAJOR, uplo, trans, diag, n, ga.t, n, gx.t, 1)
+                assert ctx.device_status() == 0
+                rx = gx.host()
+                gx.check_guards()
+                resid, scale = orc.trsv_residual(orc.ROW_MAJOR, uplo, trans, diag, n, a, n, hx, 1, rx, 1)
+                assert np.all(resid <= tol * scale), f"n={n} {uplo} {trans} {diag}: worst {np.max(resid / scale):.3e}"
+    finally:
+        b2.set_tuning(b2.KNOB_TRSV_FRONT, old[0])
+        b2.set_tuning(b2.KNOB_TRSV_CLUSTER, old[1])
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
 def test_small_integer_level2_is_bit_exact(b2, ctx, dtype):
     rng = np.random.default_rng(2)
     m, n = 300, 1100
