@@ -304,45 +304,51 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     // A thread's RS rows / columns are two chunks of V (one 16-byte pack), NB/2 apart: the packs
     // that the lanes of a warp load together then tile whole 32-byte sectors.
     // The tiles of the last two trips are inv(D_k) and inv(D_k) A_{k,k-1}, laid out in shared
-    // memory (Wt, Ms) so that the very same loads fetch them: the addresses are generic.
+    // memory (Wt, Ms) the way a matrix tile lies in global memory.
     // PM (premultiply): the last tile is replaced by inv(D_k) A_{k,k-1}, so that one product instead
     // of two stands between x_{k-1} and x_k -- at the price of two trips between x_{k-2} and
     // x_{k-1}.  It pays where the hand-over itself is slow (through L2), not inside a cluster.
     const int nm = (PM && k > 0) ? 1 : 0;
     const int yt = k - nm;  // the trip that applies inv(D_k) to b - sum
+    // full tile at base (leading dimension ld, tile origin: own rows rr0, source columns c0)
+    auto fill = [&](T (&m)[E], const T* base, int64_t ld, int64_t c0, int64_t rr0, auto ld16) {
+      if (!COLTYPE) {
+#pragma unroll
+        for (int a = 0; a < RS; ++a) {
+          const int i = (a / V) * H + V * rg + (a % V);
+          const T* src = base + (rr0 + (BACKWARD ? NB - 1 - i : i)) * ld + c0 + V * cg;
+#pragma unroll
+          for (int hb = 0; hb < RS / V; ++hb) {
+            const P pk = ld16(src + hb * H);
+#pragma unroll
+            for (int e = 0; e < V; ++e) m[a * RS + hb * V + e] = pk.v[e];
+          }
+        }
+      } else {
+#pragma unroll
+        for (int b = 0; b < RS; ++b) {
+          const int j = (b / V) * H + V * cg + (b % V);
+          const T* src = base + (c0 + j) * ld + rr0;
+#pragma unroll
+          for (int ha = 0; ha < RS / V; ++ha) {
+            const int m0 = BACKWARD ? NB - ha * H - V * rg - V : ha * H + V * rg;  // ascending memory run of the chunk
+            const P pk = ld16(src + m0);
+#pragma unroll
+            for (int e = 0; e < V; ++e) m[(ha * V + (BACKWARD ? V - 1 - e : e)) * RS + b] = pk.v[e];
+          }
+        }
+      }
+    };
     auto load_tile = [&](T (&m)[E], int s, bool raw) {
       const bool inv = !raw && s >= yt;  // trip yt reads Wt, trip k > 0 reads Ms; `raw`: the matrix tile itself
       const int64_t c0 = inv ? 0 : (int64_t)blk(s) * NB;
       const int nbJ = inv ? NB : (int)min((int64_t)NB, p.n - c0);
-      if (inv || (nbI == NB && nbJ == NB)) {
-        const T* base = inv ? (s == yt ? Wt : Ms) : p.a;
-        const int64_t ld = inv ? SP : p.lda, rr0 = inv ? 0 : r0;
-        if (!COLTYPE) {
-#pragma unroll
-          for (int a = 0; a < RS; ++a) {
-            const int i = (a / V) * H + V * rg + (a % V);
-            const T* src = base + (rr0 + (BACKWARD ? NB - 1 - i : i)) * ld + c0 + V * cg;
-#pragma unroll
-            for (int hb = 0; hb < RS / V; ++hb) {
-              const P pk = ld_generic<T, V>(src + hb * H);
-#pragma unroll
-              for (int e = 0; e < V; ++e) m[a * RS + hb * V + e] = pk.v[e];
-            }
-          }
-        } else {
-#pragma unroll
-          for (int b = 0; b < RS; ++b) {
-            const int j = (b / V) * H + V * cg + (b % V);
-            const T* src = base + (c0 + j) * ld + rr0;
-#pragma unroll
-            for (int ha = 0; ha < RS / V; ++ha) {
-              const int m0 = BACKWARD ? NB - ha * H - V * rg - V : ha * H + V * rg;  // ascending memory run of the chunk
-              const P pk = ld_generic<T, V>(src + m0);
-#pragma unroll
-              for (int e = 0; e < V; ++e) m[(ha * V + (BACKWARD ? V - 1 - e : e)) * RS + b] = pk.v[e];
-            }
-          }
-        }
+      if (inv) {
+        // (this branch runs once or twice per block row, one trip before its data is needed and
+        // before that trip waits for its x: its instruction fetches are off the critical path)
+        fill(m, s == yt ? Wt : Ms, SP, 0, 0, [](const T* q) { return *reinterpret_cast<const P*>(q); });
+      } else if (nbI == NB && nbJ == NB) {
+        fill(m, p.a, p.lda, c0, r0, [](const T* q) { return ld_nc<T, V>(q); });
       } else {
 #pragma unroll
         for (int a = 0; a < RS; ++a)
@@ -639,10 +645,13 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       const bool crit = it == k;  // the trip that ends with x_k
       const int srow = is_m ? k - 1 : it;      // the block whose x this trip multiplies (none on trip yt)
       T* xbuf_s = xs + (it & 1) * NB;
+      B2_CTRACE(ct == 0 && it == k / 2, 11);      // a trip in mid-row: start
+      B2_CTRACE(ct == 0 && it == k / 2 + 8, 12);  // eight trips later
       // first of all, off the critical path: the next tile into the other register set and a
       // tile further ahead towards L2 -- in flight while this trip waits
       if (it < k) load_tile(nxt, it + 1, false);
       prefetch_tile(it + 1 + p.pf_dist);
+      B2_CTRACE(ct == 0 && it == k / 2, 13);  // loads issued
       if (warp == 0 && !is_y) {
         const int dist = k - srow;  // rows between this block and the producer of the x
         B2_CTRACE(ct == 0 && srow == k - 1, 2);
@@ -655,6 +664,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       }
       bar_sync(kBar, kT);
       B2_CTRACE(ct == 0 && srow == k - 1 && !is_y, 8);
+      B2_CTRACE(ct == 0 && it == k / 2, 14);  // barrier passed
       const T* vec = is_y ? rbuf : xbuf_s;
       T xv[RS], part[RS];
 #pragma unroll
@@ -671,6 +681,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       }
       const T s = multi_group_sum<16, RS>(part, lane);
       B2_CTRACE(ct == 0 && srow == k - 1 && !is_y, 7);
+      B2_CTRACE(ct == 0 && it == k / 2, 15);  // reduced
       const T out = is_m ? yreg - s : s;
       if (is_y) yreg = s;
       if (it < yt) racc += s;
