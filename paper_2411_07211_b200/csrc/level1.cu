@@ -293,7 +293,10 @@ __device__ __forceinline__ void reduce_finish(typename Op::Acc acc, typename Op:
 // The arg-max reduction (iamax) instead keeps ONE running maximum per thread: a max tree per
 // chunk costs about one instruction per element, and only when a chunk raises the maximum is
 // the first element that attains it located, while the chunk is still in registers.
-template <typename T, class Op, int NV>
+// STEP = 2 serves increment 2: the kernel streams the whole span (n = its length) in 128-bit
+// packs like a unit-stride vector and lets only the even span positions count -- DRAM moves
+// whole sectors anyway, and a pack load costs a quarter of the instructions of four strided ones.
+template <typename T, class Op, int NV, int STEP = 1>
 __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__ x, const T* __restrict__ y, int64_t n,
                                                            int64_t head, int64_t nvec, int64_t nchunks,
                                                            typename Op::Acc* partials, unsigned* ticket,
@@ -303,6 +306,7 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
   using Acc = typename Op::Acc;
   const T* xv = x + head;
   const T* yv = y + head;
+  const int hp = (int)(head & 1);  // STEP 2: pack element q is a vector element iff (q & 1) == hp (V is even)
   Acc a = Op::init();
   if constexpr (Op::kArgmax) {
     T best = T(-1);
@@ -322,7 +326,7 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
         const int64_t v = v0 + (int64_t)k * kThreads;
 #pragma unroll
         for (int q = 0; q < V; ++q) {
-          px[k].v[q] = v < nvec ? fabs(px[k].v[q]) : T(-1);
+          px[k].v[q] = (v < nvec && !(STEP == 2 && ((q ^ hp) & 1))) ? fabs(px[k].v[q]) : T(-1);
           m = fmax(m, px[k].v[q]);  // fmax drops NaN operands
         }
       }
@@ -338,7 +342,7 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
     }
     if (best_chunk >= 0) {
       const int k = best_pos / V, q = best_pos % V;
-      a = Acc{best, head + (best_chunk * (int64_t)(kThreads * NV) + threadIdx.x + (int64_t)k * kThreads) * V + q};
+      a = Acc{best, (head + (best_chunk * (int64_t)(kThreads * NV) + threadIdx.x + (int64_t)k * kThreads) * V + q) / STEP};
     }
   } else {
     typename Op::Slot acc[NV][V];
@@ -359,7 +363,9 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
 #pragma unroll
         for (int k = 0; k < NV; ++k)
 #pragma unroll
-          for (int q = 0; q < V; ++q) Op::slot_accum(acc[k][q], px[k].v[q], Op::RY ? py[k].v[q] : T(0), 0);
+          for (int q = 0; q < V; ++q)
+            Op::slot_accum(acc[k][q], (STEP == 2 && ((q ^ hp) & 1)) ? T(0) : px[k].v[q],
+                           (Op::RY && !(STEP == 2 && ((q ^ hp) & 1))) ? py[k].v[q] : T(0), 0);
       } else {
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
@@ -368,7 +374,9 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
             px[k] = ld_nc<T, V>(xv + v * V);
             if (Op::RY) py[k] = ld_nc<T, V>(yv + v * V);
 #pragma unroll
-            for (int q = 0; q < V; ++q) Op::slot_accum(acc[k][q], px[k].v[q], Op::RY ? py[k].v[q] : T(0), 0);
+            for (int q = 0; q < V; ++q)
+              Op::slot_accum(acc[k][q], (STEP == 2 && ((q ^ hp) & 1)) ? T(0) : px[k].v[q],
+                           (Op::RY && !(STEP == 2 && ((q ^ hp) & 1))) ? py[k].v[q] : T(0), 0);
           }
         }
       }
@@ -384,9 +392,9 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
     int64_t i = -1;
     if ((int64_t)threadIdx.x < head) i = threadIdx.x;
     else if ((int64_t)threadIdx.x - head < ntail) i = tail0 + (threadIdx.x - head);
-    if (i >= 0) {
+    if (i >= 0 && !(STEP == 2 && (i & 1))) {
       Acc e = Op::init();
-      Op::accum(e, x[i], Op::RY ? y[i] : T(0), i);
+      Op::accum(e, x[i], Op::RY ? y[i] : T(0), i / STEP);
       a = Op::combine(a, e);
     }
   }
@@ -527,6 +535,17 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
     const int64_t grid = nchunks < 1 ? 1 : (nchunks > wave ? wave : nchunks);
     l1_reduce_unit<T, Op, NV><<<(unsigned)grid, kThreads, 0, l.stream>>>(x, Op::RY ? y : x, n, head, nvec, nchunks,
                                                                         partials, ticket, result);
+  } else if (sizeof(T) == 4 && incx == 2 && (!Op::RY || incy == 2) && same_head<T>(x, y, Op::RY, &head)) {
+    // (float only: for double, where a pack holds a single vector element, the strided kernel is the faster one)
+    constexpr int NV = Op::kPacks;
+    const int64_t span = 2 * n - 1;
+    if (head > span) head = span;
+    const int64_t nvec = (span - head) / V;
+    const int64_t nchunks = (nvec + kThreads * NV - 1) / (kThreads * NV);
+    static const int wave = one_wave(l1_reduce_unit<T, Op, NV, 2>, cap);
+    const int64_t grid = nchunks < 1 ? 1 : (nchunks > wave ? wave : nchunks);
+    l1_reduce_unit<T, Op, NV, 2><<<(unsigned)grid, kThreads, 0, l.stream>>>(x, Op::RY ? y : x, span, head, nvec, nchunks,
+                                                                           partials, ticket, result);
   } else {
     constexpr int NE = Op::RY ? 8 : 16;
     const int64_t nchunks = (n + kThreads * NE - 1) / (kThreads * NE);

@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     const int nm = (PM && k > 0) ? 1 : 0;
     const int yt = k - nm;  // the trip that applies inv(D_k) to b - sum
     // full tile at base (leading dimension ld, tile origin: own rows rr0, source columns c0)
-    auto fill = [&](T (&m)[E], const T* base, int64_t ld, int64_t c0, int64_t rr0, auto ld16) {
+    auto fill = [&](T (&m)[E], const T* base, int64_t ld, int64_t c0, int64_t rr0, bool smem) {
       if (!COLTYPE) {
 #pragma unroll
         for (int a = 0; a < RS; ++a) {
@@ -319,7 +319,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
           const T* src = base + (rr0 + (BACKWARD ? NB - 1 - i : i)) * ld + c0 + V * cg;
 #pragma unroll
           for (int hb = 0; hb < RS / V; ++hb) {
-            const P pk = ld16(src + hb * H);
+            const P pk = smem ? *reinterpret_cast<const P*>(src + hb * H) : ld_nc<T, V>(src + hb * H);
 #pragma unroll
             for (int e = 0; e < V; ++e) m[a * RS + hb * V + e] = pk.v[e];
           }
@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
 #pragma unroll
           for (int ha = 0; ha < RS / V; ++ha) {
             const int m0 = BACKWARD ? NB - ha * H - V * rg - V : ha * H + V * rg;  // ascending memory run of the chunk
-            const P pk = ld16(src + m0);
+            const P pk = smem ? *reinterpret_cast<const P*>(src + m0) : ld_nc<T, V>(src + m0);
 #pragma unroll
             for (int e = 0; e < V; ++e) m[(ha * V + (BACKWARD ? V - 1 - e : e)) * RS + b] = pk.v[e];
           }
@@ -346,9 +346,9 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       if (inv) {
         // (this branch runs once or twice per block row, one trip before its data is needed and
         // before that trip waits for its x: its instruction fetches are off the critical path)
-        fill(m, s == yt ? Wt : Ms, SP, 0, 0, [](const T* q) { return *reinterpret_cast<const P*>(q); });
+        fill(m, s == yt ? Wt : Ms, SP, 0, 0, true);
       } else if (nbI == NB && nbJ == NB) {
-        fill(m, p.a, p.lda, c0, r0, [](const T* q) { return ld_nc<T, V>(q); });
+        fill(m, p.a, p.lda, c0, r0, false);
       } else {
 #pragma unroll
         for (int a = 0; a < RS; ++a)
