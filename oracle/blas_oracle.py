@@ -154,6 +154,20 @@ def ger(order, m, n, alpha, x, incx, y, incy, a, lda, want_absterms=True):
     return None if absterms is None else absterms.reshape(m, n)
 
 
+def syr(order, uplo, n, alpha, x, incx, a, lda, want_absterms=True):
+    absterms = np.zeros(n * n, dtype=np.float64) if want_absterms else None
+    _call("syr", a.dtype, _int(order), _int(uplo), _i64(n), _scalar(a.dtype, alpha), _ptr(x), _i64(incx),
+          _ptr(a), _i64(lda), _ptr(absterms))
+    return None if absterms is None else absterms.reshape(n, n)
+
+
+def syr2(order, uplo, n, alpha, x, incx, y, incy, a, lda, want_absterms=True):
+    absterms = np.zeros(n * n, dtype=np.float64) if want_absterms else None
+    _call("syr2", a.dtype, _int(order), _int(uplo), _i64(n), _scalar(a.dtype, alpha), _ptr(x), _i64(incx),
+          _ptr(y), _i64(incy), _ptr(a), _i64(lda), _ptr(absterms))
+    return None if absterms is None else absterms.reshape(n, n)
+
+
 def symv(order, uplo, n, alpha, a, lda, x, incx, beta, y, incy):
     absterms = np.zeros(n, dtype=np.float64)
     _call("symv", a.dtype, _int(order), _int(uplo), _i64(n), _scalar(a.dtype, alpha), _ptr(a),

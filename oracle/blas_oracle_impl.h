@@ -196,6 +196,50 @@ void FN(ger)(int order, int64_t m, int64_t n, T alpha, const T* x, int64_t incx,
   }
 }
 
+/* syr: A[i,j] += alpha * x[i] * x[j] for the (i,j) of the uplo triangle (121 upper: i <= j,
+ * 122 lower: i >= j), A symmetric n x n with that triangle stored; the other triangle is never
+ * touched.  alpha == 0 leaves A untouched.  One of the symmetric rank-1 updates of Section 6.2.2
+ * ("symmetric rank-1 update"); the BLAS problem statement the paper adopts defines it.
+ * absterms (optional) is a dense n*n array in (i*n + j) order; entries outside the triangle
+ * are left as they are. */
+void FN(syr)(int order, int uplo, int64_t n, T alpha, const T* x, int64_t incx, T* a, int64_t lda,
+             double* absterms) {
+  for (int64_t i = 0; i < n; ++i) {
+    for (int64_t j = 0; j < n; ++j) {
+      int stored = uplo == 121 ? (i <= j) : (i >= j);
+      if (!stored) continue;
+      W aij = (W)a[MIDX(order, i, j, lda)];
+      if (alpha == (T)0) {
+        if (absterms) absterms[i * n + j] = (double)WABS(aij);
+        continue;
+      }
+      W p = (W)alpha * ((W)x[VIDX(i, n, incx)] * (W)x[VIDX(j, n, incx)]);
+      a[MIDX(order, i, j, lda)] = (T)(p + aij);
+      if (absterms) absterms[i * n + j] = (double)(WABS(p) + WABS(aij));
+    }
+  }
+}
+
+/* syr2: A[i,j] += alpha * (x[i]*y[j] + y[i]*x[j]) on the uplo triangle; same conventions as syr. */
+void FN(syr2)(int order, int uplo, int64_t n, T alpha, const T* x, int64_t incx, const T* y,
+              int64_t incy, T* a, int64_t lda, double* absterms) {
+  for (int64_t i = 0; i < n; ++i) {
+    for (int64_t j = 0; j < n; ++j) {
+      int stored = uplo == 121 ? (i <= j) : (i >= j);
+      if (!stored) continue;
+      W aij = (W)a[MIDX(order, i, j, lda)];
+      if (alpha == (T)0) {
+        if (absterms) absterms[i * n + j] = (double)WABS(aij);
+        continue;
+      }
+      W p1 = (W)alpha * ((W)x[VIDX(i, n, incx)] * (W)y[VIDX(j, n, incy)]);
+      W p2 = (W)alpha * ((W)y[VIDX(i, n, incy)] * (W)x[VIDX(j, n, incx)]);
+      a[MIDX(order, i, j, lda)] = (T)(p1 + p2 + aij);
+      if (absterms) absterms[i * n + j] = (double)(WABS(p1) + WABS(p2) + WABS(aij));
+    }
+  }
+}
+
 /* Element (i,j) of a symmetric matrix of which only the uplo triangle is stored
  * (121 upper: i <= j stored, 122 lower: i >= j stored).  The other triangle is never read. */
 static inline W OR_CAT(P, _sym_elem)(int order, int uplo, const T* a, int64_t lda, int64_t i,

@@ -475,3 +475,83 @@ def test_golden_sdot_config1():
     # independent evaluation: numpy pairwise float64 sum of exact float64 products
     ref = np.sum(x.astype(np.float64) * y.astype(np.float64))
     assert abs(float(res) - ref) <= 2.0 ** -24 * abs(ref) + 1e-9 * absterms
+
+
+# ----------------------------------------------------------------- syr / syr2 (the "next" rows)
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("order", ORDERS)
+@pytest.mark.parametrize("uplo", UPLOS)
+@pytest.mark.parametrize("n,pad", [(1, 0), (2, 1), (5, 0), (8, 3)])
+def test_syr_syr2_bruteforce(dtype, order, uplo, n, pad):
+    """Exact rational evaluation of the definition on the stored triangle; the other triangle,
+    the pad columns and the strided gaps are NaN and must stay untouched / unread."""
+    lda = n + pad
+    a = _tri_buf(11, n, lda, dtype, order, uplo, orc.NON_UNIT)
+    dense = dense_full(order, n, n, a, lda)
+    alpha = dtype(1.25)
+    fa = Fraction(float(alpha))
+    for incx, incy in [(1, 1), (2, 3), (-1, 2)]:
+        x, y = rand(3, n, n, dtype), rand(4, n + 1, n, dtype)
+        fx, fy = fr(x), fr(y)
+        for two in (False, True):
+            a2 = a.copy()
+            if two:
+                absterms = orc.syr2(order, uplo, n, alpha, strided(x, incx), incx, strided(y, incy), incy, a2, lda)
+            else:
+                absterms = orc.syr(order, uplo, n, alpha, strided(x, incx), incx, a2, lda)
+            got = dense_full(order, n, n, a2, lda)
+            for i in range(n):
+                for j in range(n):
+                    inside = (i <= j) if uplo == orc.UPPER else (i >= j)
+                    if not inside:
+                        assert np.isnan(got[i][j])  # never written
+                        continue
+                    upd = fa * (fx[i] * fy[j] + fy[i] * fx[j]) if two else fa * fx[i] * fx[j]
+                    assert_within_ulp(np.array([got[i][j]], dtype=dtype), [upd + Fraction(float(dense[i][j]))], dtype)
+                    terms = ([abs(fa * fx[i] * fy[j]), abs(fa * fy[i] * fx[j])] if two else [abs(fa * fx[i] * fx[j])])
+                    want_abs = float(sum(terms) + abs(Fraction(float(dense[i][j]))))
+                    assert np.isclose(absterms[i, j], want_abs, rtol=1e-12)
+            assert np.isnan(a2).sum() == np.isnan(a).sum()
+            a3 = a.copy()  # alpha == 0: untouched, vectors never matter
+            nanx = np.full_like(strided(x, incx), np.nan)
+            if two:
+                orc.syr2(order, uplo, n, dtype(0), nanx, incx, np.full_like(strided(y, incy), np.nan), incy, a3, lda)
+            else:
+                orc.syr(order, uplo, n, dtype(0), nanx, incx, a3, lda)
+            assert np.array_equal(a3, a, equal_nan=True)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("uplo", UPLOS)
+def test_syr_invariants(dtype, uplo):
+    """syr equals ger(x, x) on the triangle; syr2(x, x) with alpha equals syr with 2*alpha (exact:
+    a power of two); row-major upper equals column-major lower on the same buffer; from A = 0
+    the result is alpha*x_i*x_j."""
+    n = 37
+    x, y = rand(5, n, n, dtype), rand(6, n, n, dtype)
+    full = synth.matrix_np(9, 2, n, n, n, dtype).ravel()
+    alpha = dtype(0.75)
+    g = full.copy()
+    orc.ger(orc.ROW_MAJOR, n, n, alpha, x, 1, x, 1, g, n, want_absterms=False)
+    s1 = full.copy()
+    orc.syr(orc.ROW_MAJOR, uplo, n, alpha, x, 1, s1, n, want_absterms=False)
+    r, c = np.indices((n, n))
+    inside = ((r <= c) if uplo == orc.UPPER else (r >= c)).ravel()
+    assert np.array_equal(s1[inside], g[inside]) and np.array_equal(s1[~inside], full[~inside])
+    s2 = full.copy()
+    orc.syr2(orc.ROW_MAJOR, uplo, n, alpha, x, 1, x, 1, s2, n, want_absterms=False)
+    s3 = full.copy()
+    orc.syr(orc.ROW_MAJOR, uplo, n, dtype(2) * alpha, x, 1, s3, n, want_absterms=False)
+    tol = 4 * np.finfo(dtype).eps
+    assert np.all(np.abs(s2 - s3) <= tol * (np.abs(s3) + 1))
+    other = orc.LOWER if uplo == orc.UPPER else orc.UPPER
+    s4 = full.copy()
+    orc.syr2(orc.COL_MAJOR, other, n, alpha, x, 1, y, 1, s4, n, want_absterms=False)
+    s5 = full.copy()
+    orc.syr2(orc.ROW_MAJOR, uplo, n, alpha, x, 1, y, 1, s5, n, want_absterms=False)
+    assert np.array_equal(s4, s5)
+    z = np.zeros(n * n, dtype=dtype)
+    orc.syr(orc.ROW_MAJOR, uplo, n, alpha, x, 1, z, n, want_absterms=False)
+    want = (np.longdouble(alpha) * np.outer(x.astype(np.longdouble), x.astype(np.longdouble))).ravel()
+    err = np.abs(z.astype(np.longdouble) - want)[inside]
+    assert np.all(err <= np.spacing(np.abs(z[inside])).astype(np.longdouble)) and np.all(z[~inside] == 0)
