@@ -161,6 +161,21 @@ int b2_sger(const b2_ctx* ctx, int order, int64_t m, int64_t n, float alpha, con
 int b2_dger(const b2_ctx* ctx, int order, int64_t m, int64_t n, double alpha, const double* x, int64_t incx,
             const double* y, int64_t incy, double* a, int64_t lda);
 
+/* syr (Section 6.2.2, "symmetric rank-1 update"): A <- alpha*x*x^T + A on the uplo triangle
+ * (with the diagonal) of the symmetric n x n matrix A; the other triangle is neither read nor
+ * written.  alpha == 0: no-op.  Elementwise two-term sums: same tolerance class as ger. */
+int b2_ssyr(const b2_ctx* ctx, int order, int uplo, int64_t n, float alpha, const float* x, int64_t incx, float* a,
+            int64_t lda);
+int b2_dsyr(const b2_ctx* ctx, int order, int uplo, int64_t n, double alpha, const double* x, int64_t incx, double* a,
+            int64_t lda);
+
+/* syr2 (Section 6.2.2, "symmetric rank-2 update"): A <- alpha*(x*y^T + y*x^T) + A on the uplo
+ * triangle; otherwise as syr. */
+int b2_ssyr2(const b2_ctx* ctx, int order, int uplo, int64_t n, float alpha, const float* x, int64_t incx,
+             const float* y, int64_t incy, float* a, int64_t lda);
+int b2_dsyr2(const b2_ctx* ctx, int order, int uplo, int64_t n, double alpha, const double* x, int64_t incx,
+             const double* y, int64_t incy, double* a, int64_t lda);
+
 /* symv: y <- alpha*A*x + beta*y, A symmetric n x n; only the uplo triangle (with the
  * diagonal) is referenced, the other triangle is never used. */
 int b2_ssymv(const b2_ctx* ctx, int order, int uplo, int64_t n, float alpha, const float* a, int64_t lda,

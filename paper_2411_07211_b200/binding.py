@@ -63,6 +63,8 @@ def _protos():
         out[f"b2_{p}gemv"] = [cp, _int, _int, _i64, _i64, sc, _vp, _i64, _vp, _i64, sc, _vp, _i64]
         out[f"b2_{p}ger"] = [cp, _int, _i64, _i64, sc, _vp, _i64, _vp, _i64, _vp, _i64]
         out[f"b2_{p}symv"] = [cp, _int, _int, _i64, sc, _vp, _i64, _vp, _i64, sc, _vp, _i64]
+        out[f"b2_{p}syr"] = [cp, _int, _int, _i64, sc, _vp, _i64, _vp, _i64]
+        out[f"b2_{p}syr2"] = [cp, _int, _int, _i64, sc, _vp, _i64, _vp, _i64, _vp, _i64]
         out[f"b2_{p}trmv"] = [cp, _int, _int, _int, _int, _i64, _vp, _i64, _vp, _i64]
         out[f"b2_{p}trsv"] = [cp, _int, _int, _int, _int, _i64, _vp, _i64, _vp, _i64]
     out["b2_sdot_noalloc"] = [_vp, _i64, _vp, _i64, _vp, _i64, _vp]
@@ -205,6 +207,15 @@ def gemv(ctx, order, trans, m, n, alpha, a, lda, x, incx, beta, y, incy, check=T
 
 def ger(ctx, order, m, n, alpha, x, incx, y, incy, a, lda, check=True):
     return _call(f"b2_{_prefix(a)}ger", ctx, order, m, n, alpha, _p(x), incx, _p(y), incy, _p(a), lda, check=check)
+
+
+def syr(ctx, order, uplo, n, alpha, x, incx, a, lda, check=True):
+    return _call(f"b2_{_prefix(a)}syr", ctx, order, uplo, n, alpha, _p(x), incx, _p(a), lda, check=check)
+
+
+def syr2(ctx, order, uplo, n, alpha, x, incx, y, incy, a, lda, check=True):
+    return _call(f"b2_{_prefix(a)}syr2", ctx, order, uplo, n, alpha, _p(x), incx, _p(y), incy, _p(a), lda,
+                 check=check)
 
 
 def symv(ctx, order, uplo, n, alpha, a, lda, x, incx, beta, y, incy, check=True):

@@ -15,7 +15,7 @@ INCLUDE = os.path.join(ROOT, "include")
 OBJ_DIR = os.path.join(PKG, "_build")
 LIB_PATH = os.path.join(PKG, "libb2blas.so")
 
-SOURCES = ["api_common.cu", "level1.cu", "gemv.cu", "ger.cu", "tri_f32.cu", "tri_f64.cu", "trsv.cu", "trsv_front.cu"]
+SOURCES = ["api_common.cu", "level1.cu", "gemv.cu", "ger.cu", "tri_f32.cu", "tri_f64.cu", "trsv.cu", "trsv_front.cu", "syr.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 
