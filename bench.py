@@ -240,6 +240,45 @@ class GpuWorkload:
                 events[k][1].record()
 
 
+def next_rows_leg(wl: GpuWorkload, steps: int, peak: float):
+    """The routines beyond the 14 of the headline metric (built after them: syr, syr2), timed the
+    same way (L2 swept, one event bracket per call, median) on a 256 MiB working set; they are NOT
+    part of `value`.  They update the general matrix of the ger variants in place: this leg runs
+    after everything else."""
+    torch, b2, ctx, B = wl.torch, wl.b2, wl.ctx, wl.buf
+    rows = []
+    for dt, s in (("f32", 4), ("f64", 8)):
+        if (dt, "ager") not in B:
+            continue
+        n = 8192 if s == 4 else 5760
+        tri = n * (n + 1) // 2
+        for r in ("syr", "syr2"):
+            for ul, un in ((UP, "u"), (LO, "l")):
+                for inc in (1, 2):
+                    ts = []
+                    for it in range(steps + 3):
+                        wl.sweep_l2()
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                        if r == "syr":
+                            b2.syr(ctx, ROW, ul, n, 1e-3, B[dt, "vx0"], inc, B[dt, "ager"], n)
+                        else:
+                            b2.syr2(ctx, ROW, ul, n, 1e-3, B[dt, "vx0"], inc, B[dt, "vy0"], inc, B[dt, "ager"], n)
+                        e1.record()
+                        torch.cuda.synchronize()
+                        if it >= 3:
+                            ts.append(e0.elapsed_time(e1))
+                    ts.sort()
+                    ms = ts[len(ts) // 2]
+                    nvec = 1 if r == "syr" else 2
+                    touched = 2 * tri * s + nvec * n * s * inc
+                    gbs = touched / (ms * 1e-3) / 1e9
+                    rows.append({"name": f"{r}_{un}_{dt}_inc{inc}", "ms": round(ms, 4), "gbs": round(gbs, 1),
+                                 "frac": round(gbs / peak, 4)})
+    return {"note": "rows built after the headline set; bytes = 2 x stored triangle + vectors; not part of `value`",
+            "geomean_frac": geomean([r["frac"] for r in rows]), "variants": rows}
+
+
 def e2e_leg(wl: GpuWorkload, steps: int):
     """Same metric through the C ABI with HOST data: per variant, pinned host -> device copies of
     its inputs, the call, and a device -> host read of its outputs, all inside the timed bracket."""
@@ -529,6 +568,8 @@ def main():
     else:
         out["cpu_baseline"] = None
     out["variants"] = [{k: (round(v, 4) if isinstance(v, float) else v) for k, v in r.items()} for r in rows]
+    if world == 1 and not args.filter:
+        out["next_rows"] = next_rows_leg(wl, min(args.steps, 10), peak)
     if args.table:
         os.makedirs(os.path.dirname(os.path.abspath(args.table)), exist_ok=True)
         with open(args.table, "w") as f:
