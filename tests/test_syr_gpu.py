@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 DTYPES = [np.float32, np.float64]
 ORDERS = [orc.ROW_MAJOR, orc.COL_MAJOR]
 UPLOS = [orc.UPPER, orc.LOWER]
-SIZES = [1, 2, 5, 31, 64, 65, 127, 257, 300, 1100]
+SIZES = [1, 2, 5, 31, 64, 65, 127, 257, 300, 1100, 1537]
 
 
 @pytest.fixture(scope="module")
