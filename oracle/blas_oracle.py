@@ -109,6 +109,38 @@ def rot(n, x, incx, y, incy, c, s):
     return ax, ay
 
 
+def rotm(n, x, incx, y, incy, param):
+    """param = [flag, h11, h21, h12, h22] (numpy, same dtype as x); returns absterms of x' and y'."""
+    ax = np.zeros(n, dtype=np.float64)
+    ay = np.zeros(n, dtype=np.float64)
+    param = np.ascontiguousarray(param, dtype=x.dtype)
+    assert param.shape == (5,)
+    _call("rotm", x.dtype, _i64(n), _ptr(x), _i64(incx), _ptr(y), _i64(incy), _ptr(param), _ptr(ax), _ptr(ay))
+    return ax, ay
+
+
+def dsdot(n, x, incx, y, incy):
+    """float32 inputs, double result."""
+    assert x.dtype == np.float32 and y.dtype == np.float32
+    res = np.zeros(1, dtype=np.float64)
+    absterms = np.zeros(1, dtype=np.float64)
+    f = lib().oracle_dsdot
+    f.restype = None
+    f(_i64(n), _ptr(x), _i64(incx), _ptr(y), _i64(incy), _ptr(res), _ptr(absterms))
+    return res[0], absterms[0]
+
+
+def sdsdot(n, sb, x, incx, y, incy):
+    """float32 inputs, float32 result = sb + the double-accumulated dot."""
+    assert x.dtype == np.float32 and y.dtype == np.float32
+    res = np.zeros(1, dtype=np.float32)
+    absterms = np.zeros(1, dtype=np.float64)
+    f = lib().oracle_sdsdot
+    f.restype = None
+    f(_i64(n), ctypes.c_float(sb), _ptr(x), _i64(incx), _ptr(y), _i64(incy), _ptr(res), _ptr(absterms))
+    return res[0], absterms[0]
+
+
 def dot(n, x, incx, y, incy):
     res = np.zeros(1, dtype=x.dtype)
     absterms = np.zeros(1, dtype=np.float64)

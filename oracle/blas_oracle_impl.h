@@ -97,6 +97,39 @@ void FN(rot)(int64_t n, T* x, int64_t incx, T* y, int64_t incy, T c, T s,
   }
 }
 
+/* rotm: the modified Givens rotation (the paper's level-1 set, Section 6.2.1, includes rotm;
+ * the definition is the BLAS one).  (x_i, y_i) <- (h11 x_i + h12 y_i, h21 x_i + h22 y_i), both
+ * from the old pair, with H selected by flag = param[0]:
+ *   flag = -1 : H = [h11 h12; h21 h22]   all four from param
+ *   flag =  0 : H = [  1 h12; h21   1]   the diagonal is implied, param[1] and param[4] unread
+ *   flag =  1 : H = [h11   1;  -1 h22]   the off-diagonal is implied, param[2] and param[3] unread
+ *   flag = -2 : H = I                    nothing is read or written
+ * param = {flag, h11, h21, h12, h22}.  An implied 1 or -1 means no multiplication: that term is
+ * the element itself (or its negation). */
+void FN(rotm)(int64_t n, T* x, int64_t incx, T* y, int64_t incy, const T* param,
+              double* absterms_x, double* absterms_y) {
+  const T flag = param[0];
+  if (flag == (T)-2) return;
+  for (int64_t i = 0; i < n; ++i) {
+    W xi = (W)x[VIDX(i, n, incx)], yi = (W)y[VIDX(i, n, incy)];
+    W xx, xy, yx, yy; /* the four terms: x' = xx + xy, y' = yx + yy */
+    if (flag == (T)-1) {
+      xx = (W)param[1] * xi; xy = (W)param[3] * yi;
+      yx = (W)param[2] * xi; yy = (W)param[4] * yi;
+    } else if (flag == (T)0) {
+      xx = xi;               xy = (W)param[3] * yi;
+      yx = (W)param[2] * xi; yy = yi;
+    } else { /* flag == 1 */
+      xx = (W)param[1] * xi; xy = yi;
+      yx = -xi;              yy = (W)param[4] * yi;
+    }
+    x[VIDX(i, n, incx)] = (T)(xx + xy);
+    y[VIDX(i, n, incy)] = (T)(yx + yy);
+    if (absterms_x) absterms_x[i] = (double)(WABS(xx) + WABS(xy));
+    if (absterms_y) absterms_y[i] = (double)(WABS(yx) + WABS(yy));
+  }
+}
+
 /* dot: sum_i x_i y_i. */
 void FN(dot)(int64_t n, const T* x, int64_t incx, const T* y, int64_t incy, T* result,
              double* absterms) {

@@ -555,3 +555,118 @@ def test_syr_invariants(dtype, uplo):
     want = (np.longdouble(alpha) * np.outer(x.astype(np.longdouble), x.astype(np.longdouble))).ravel()
     err = np.abs(z.astype(np.longdouble) - want)[inside]
     assert np.all(err <= np.spacing(np.abs(z[inside])).astype(np.longdouble)) and np.all(z[~inside] == 0)
+
+
+# ----------------------------------------------------------------- rotm / dsdot / sdsdot (the "next" rows)
+def _h_of(flag, h11, h21, h12, h22):
+    """The 2x2 matrix the flag selects, as exact rationals (BLAS definition of rotm)."""
+    one = Fraction(1)
+    f = lambda v: Fraction(float(v))
+    if flag == -1:
+        return f(h11), f(h12), f(h21), f(h22)
+    if flag == 0:
+        return one, f(h12), f(h21), one
+    if flag == 1:
+        return f(h11), one, -one, f(h22)
+    return one, Fraction(0), Fraction(0), one
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("flag", [-2, -1, 0, 1])
+@pytest.mark.parametrize("n", [1, 3, 8])
+@pytest.mark.parametrize("incx,incy", [(1, 1), (2, -1), (-3, 2)])
+def test_rotm_bruteforce(dtype, flag, n, incx, incy):
+    x, y = rand(5, 30 + n, n, dtype), rand(5, 40 + n, n, dtype)
+    fx, fy = fr(x), fr(y)
+    h11, h21, h12, h22 = dtype(0.75), dtype(-1.3), dtype(0.4), dtype(1.7)
+    a11, a12, a21, a22 = _h_of(flag, h11, h21, h12, h22)
+    # the entries the flag implies must not be read: poison them
+    param = np.array([flag, h11, h21, h12, h22], dtype=dtype)
+    if flag == 0:
+        param[1] = param[4] = np.nan
+    if flag == 1:
+        param[2] = param[3] = np.nan
+    if flag == -2:
+        param[1:] = np.nan
+    bx, by = strided(x, incx), strided(y, incy)
+    ax, ay = orc.rotm(n, bx, incx, by, incy, param)
+    if flag == -2:  # identity: bit-for-bit untouched
+        assert np.array_equal(bx, strided(x, incx), equal_nan=True)
+        assert np.array_equal(by, strided(y, incy), equal_nan=True)
+        return
+    assert_within_ulp(logical(bx, n, incx), [a11 * a + a12 * b for a, b in zip(fx, fy)], dtype)
+    assert_within_ulp(logical(by, n, incy), [a21 * a + a22 * b for a, b in zip(fx, fy)], dtype)
+    assert np.allclose(ax, [float(abs(a11 * a) + abs(a12 * b)) for a, b in zip(fx, fy)], rtol=1e-12)
+    assert np.allclose(ay, [float(abs(a21 * a) + abs(a22 * b)) for a, b in zip(fx, fy)], rtol=1e-12)
+    assert np.isnan(bx).sum() == np.isnan(strided(x, incx)).sum()  # gaps untouched
+    assert np.isnan(by).sum() == np.isnan(strided(y, incy)).sum()
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_rotm_reduces_to_rot_and_to_explicit_h(dtype):
+    """flag -1 with H = [c s; -s c] is the plain rotation (pinned above) bit for bit; flags 0 and 1
+    equal flag -1 with the implied entries written out; two rotm's compose like the matrix product
+    on exactly representable data."""
+    n = 37
+    x, y = rand(6, 1, n, dtype), rand(6, 2, n, dtype)
+    c, s = dtype(0.6), dtype(0.8)
+    x1, y1, x2, y2 = x.copy(), y.copy(), x.copy(), y.copy()
+    orc.rot(n, x1, 1, y1, 1, c, s)
+    orc.rotm(n, x2, 1, y2, 1, np.array([-1, c, -s, s, c], dtype=dtype))
+    assert np.array_equal(x1, x2) and np.array_equal(y1, y2)
+    h11, h21, h12, h22 = dtype(0.5), dtype(-0.25), dtype(1.5), dtype(2.0)
+    for flag, full in ((0, [-1, 1, h21, h12, 1]), (1, [-1, h11, -1, 1, h22])):
+        x1, y1, x2, y2 = x.copy(), y.copy(), x.copy(), y.copy()
+        orc.rotm(n, x1, 1, y1, 1, np.array([flag, h11, h21, h12, h22], dtype=dtype))
+        orc.rotm(n, x2, 1, y2, 1, np.array(full, dtype=dtype))
+        assert np.array_equal(x1, x2) and np.array_equal(y1, y2)
+    # exact data (small integers, dyadic H): H2 (H1 v) == (H2 H1) v with no rounding anywhere
+    xi = np.arange(-18, 19, dtype=dtype)
+    yi = np.arange(37, 0, -1, dtype=dtype)
+    h1 = np.array([[0.5, 1.5], [-0.25, 2.0]])
+    h2 = np.array([[2.0, -0.5], [0.75, 1.0]])
+    xa, ya = xi.copy(), yi.copy()
+    orc.rotm(n, xa, 1, ya, 1, np.array([-1, h1[0, 0], h1[1, 0], h1[0, 1], h1[1, 1]], dtype=dtype))
+    orc.rotm(n, xa, 1, ya, 1, np.array([-1, h2[0, 0], h2[1, 0], h2[0, 1], h2[1, 1]], dtype=dtype))
+    h = h2 @ h1
+    assert np.array_equal(xa, (h[0, 0] * xi + h[0, 1] * yi).astype(dtype))
+    assert np.array_equal(ya, (h[1, 0] * xi + h[1, 1] * yi).astype(dtype))
+
+
+@pytest.mark.parametrize("n", [0, 1, 2, 5, 8])
+@pytest.mark.parametrize("incx,incy", [(1, 1), (2, 1), (-1, 3), (-2, -1)])
+def test_dsdot_sdsdot_bruteforce(n, incx, incy):
+    x, y = rand(7, 50 + n, n, np.float32), rand(7, 60 + n, n, np.float32)
+    fx, fy = fr(x), fr(y)
+    exact = sum((a * b for a, b in zip(fx, fy)), Fraction(0))
+    bx, by = strided(x, incx), strided(y, incy)
+    d, dabs = orc.dsdot(n, bx, incx, by, incy)
+    assert isinstance(d, np.float64)
+    assert_within_ulp(d, [exact], np.float64)
+    assert np.isclose(dabs, float(sum((abs(a * b) for a, b in zip(fx, fy)), Fraction(0))), rtol=1e-12)
+    sb = np.float32(-0.3125)
+    r, rabs = orc.sdsdot(n, sb, bx, incx, by, incy)
+    assert isinstance(r, np.float32)
+    assert_within_ulp(r, [exact + Fraction(float(sb))], np.float32)
+    assert np.isclose(rabs, dabs + abs(float(sb)), rtol=1e-12)
+
+
+def test_dsdot_keeps_what_float_accumulation_loses():
+    """Cancellation that a float accumulator cannot survive: 2^30*1 + 1*1 - 2^30*1 is exactly 1;
+    in float 2^30 + 1 rounds to 2^30 and the sum would be 0.  Also: dsdot equals the double dot
+    product of the widened inputs (products of floats are exact in double)."""
+    x = np.array([2.0 ** 30, 1.0, -(2.0 ** 30)], dtype=np.float32)
+    y = np.ones(3, dtype=np.float32)
+    assert np.float32(np.float32(2.0 ** 30) + np.float32(1.0)) == np.float32(2.0 ** 30)
+    assert orc.dsdot(3, x, 1, y, 1)[0] == 1.0
+    assert orc.sdsdot(3, np.float32(0.5), x, 1, y, 1)[0] == np.float32(1.5)
+    # a sum whose exact value needs more than 24 bits: 2^24 + 1 is not a float, but is a double
+    x = np.array([2.0 ** 12, 1.0], dtype=np.float32)
+    y = np.array([2.0 ** 12, 1.0], dtype=np.float32)
+    assert orc.dsdot(2, x, 1, y, 1)[0] == 2.0 ** 24 + 1
+    assert orc.sdsdot(2, np.float32(0), x, 1, y, 1)[0] == np.float32(2.0 ** 24)  # ties-to-even
+    n = 1000
+    x, y = rand(8, 1, n, np.float32), rand(8, 2, n, np.float32)
+    wide = orc.dot(n, x.astype(np.float64), 1, y.astype(np.float64), 1)[0]
+    assert orc.dsdot(n, x, 1, y, 1)[0] == wide
+    assert abs(wide - np.dot(x.astype(np.float64), y.astype(np.float64))) <= 1e-13 * float(np.sum(np.abs(x * y)))
