@@ -110,9 +110,28 @@ int b2_dswap(const b2_ctx* ctx, int64_t n, double* x, int64_t incx, double* y, i
 int b2_srot(const b2_ctx* ctx, int64_t n, float* x, int64_t incx, float* y, int64_t incy, float c, float s);
 int b2_drot(const b2_ctx* ctx, int64_t n, double* x, int64_t incx, double* y, int64_t incy, double c, double s);
 
+/* rotm (Section 6.2.1 lists rotm among the level-1 kernels; the definition is the BLAS one):
+ * the modified Givens rotation (x_i, y_i) <- (h11*x_i + h12*y_i, h21*x_i + h22*y_i).
+ *   param   HOST pointer to 5 values {flag, h11, h21, h12, h22}; it is read before the call
+ *           returns.  flag -1: all four entries from param; flag 0: h11 = h22 = 1 implied
+ *           (param[1], param[4] not read); flag 1: h12 = 1, h21 = -1 implied (param[2],
+ *           param[3] not read); flag -2: H = I, nothing is launched.
+ * Errors: -1 n, -2 x, -3 incx, -4 y, -5 incy, -6 param (NULL or a flag outside {-2,-1,0,1}). */
+int b2_srotm(const b2_ctx* ctx, int64_t n, float* x, int64_t incx, float* y, int64_t incy, const float* param);
+int b2_drotm(const b2_ctx* ctx, int64_t n, double* x, int64_t incx, double* y, int64_t incy, const double* param);
+
 /* dot: *result <- sum_i x_i*y_i.  Reductions are deterministic: same inputs, same bits. */
 int b2_sdot(const b2_ctx* ctx, int64_t n, const float* x, int64_t incx, const float* y, int64_t incy, float* result);
 int b2_ddot(const b2_ctx* ctx, int64_t n, const double* x, int64_t incx, const double* y, int64_t incy, double* result);
+
+/* dsdot (Section 6.2.1 lists dsdot among the level-1 kernels): float vectors, every product and
+ * the sum in double: *result <- sum_i (double)x_i * (double)y_i, a DEVICE double.
+ * sdsdot: *result <- (float)(sb + that double sum), a DEVICE float, rounded once; it keeps the
+ * double sum in ctx->workspace behind the block partials and runs one extra one-thread kernel.
+ * Errors: dsdot as b2_sdot; sdsdot -1 n, -3 x, -4 incx, -5 y, -6 incy, -7 result. */
+int b2_dsdot(const b2_ctx* ctx, int64_t n, const float* x, int64_t incx, const float* y, int64_t incy, double* result);
+int b2_sdsdot(const b2_ctx* ctx, int64_t n, float sb, const float* x, int64_t incx, const float* y, int64_t incy,
+              float* result);
 
 /* sdot without any caller-provided or allocated scratch (the paper has no counterpart: this
  * entry point exists for deployment reasons only).  Same result contract as b2_sdot, but no

@@ -56,6 +56,7 @@ def _protos():
         out[f"b2_{p}copy"] = [cp, _i64, _vp, _i64, _vp, _i64]
         out[f"b2_{p}swap"] = [cp, _i64, _vp, _i64, _vp, _i64]
         out[f"b2_{p}rot"] = [cp, _i64, _vp, _i64, _vp, _i64, sc, sc]
+        out[f"b2_{p}rotm"] = [cp, _i64, _vp, _i64, _vp, _i64, _vp]
         out[f"b2_{p}dot"] = [cp, _i64, _vp, _i64, _vp, _i64, _vp]
         out[f"b2_{p}asum"] = [cp, _i64, _vp, _i64, _vp]
         out[f"b2_{p}nrm2"] = [cp, _i64, _vp, _i64, _vp]
@@ -67,6 +68,8 @@ def _protos():
         out[f"b2_{p}syr2"] = [cp, _int, _int, _i64, sc, _vp, _i64, _vp, _i64, _vp, _i64]
         out[f"b2_{p}trmv"] = [cp, _int, _int, _int, _int, _i64, _vp, _i64, _vp, _i64]
         out[f"b2_{p}trsv"] = [cp, _int, _int, _int, _int, _i64, _vp, _i64, _vp, _i64]
+    out["b2_dsdot"] = [cp, _i64, _vp, _i64, _vp, _i64, _vp]
+    out["b2_sdsdot"] = [cp, _i64, _f, _vp, _i64, _vp, _i64, _vp]
     out["b2_sdot_noalloc"] = [_vp, _i64, _vp, _i64, _vp, _i64, _vp]
     out["b2_workspace_reset"] = [cp]
     return out
@@ -181,6 +184,25 @@ def swap(ctx, n, x, incx, y, incy, check=True):
 
 def rot(ctx, n, x, incx, y, incy, c, s, check=True):
     return _call(f"b2_{_prefix(x)}rot", ctx, n, _p(x), incx, _p(y), incy, c, s, check=check)
+
+
+def rotm(ctx, n, x, incx, y, incy, param, check=True):
+    """param: 5 host values [flag, h11, h21, h12, h22] (any sequence); None passes a NULL pointer."""
+    if param is None:
+        hp = None
+    else:
+        ctype = ctypes.c_float if x.dtype == torch.float32 else ctypes.c_double
+        hp = ctypes.cast((ctype * 5)(*[float(v) for v in param]), _vp)
+    return _call(f"b2_{_prefix(x)}rotm", ctx, n, _p(x), incx, _p(y), incy, hp, check=check)
+
+
+def dsdot(ctx, n, x, incx, y, incy, result, check=True):
+    """float32 vectors, float64 device result."""
+    return _call("b2_dsdot", ctx, n, _p(x), incx, _p(y), incy, _p(result), check=check)
+
+
+def sdsdot(ctx, n, sb, x, incx, y, incy, result, check=True):
+    return _call("b2_sdsdot", ctx, n, sb, _p(x), incx, _p(y), incy, _p(result), check=check)
 
 
 def dot(ctx, n, x, incx, y, incy, result, check=True):

@@ -53,6 +53,21 @@ struct RotOp {
   }
 };
 
+// Modified Givens rotation: (x, y) <- (h11 x + h12 y, h21 x + h22 y).  The host has already
+// written the entries the flag implies (1, -1) into the four coefficients; a product with
+// +-1 is exact, so the implied forms lose nothing against skipping the multiplication.
+template <typename T>
+struct RotmOp {
+  T h11, h12, h21, h22;
+  static constexpr bool RX = true, RY = true, WX = true, WY = true;
+  __device__ __forceinline__ void operator()(T& x, T& y) const {
+    T nx = h11 * x + h12 * y;
+    T ny = h21 * x + h22 * y;
+    x = nx;
+    y = ny;
+  }
+};
+
 // Unit stride.  The vector region is [head, head + nvec*V); up to V-1 head and V-1 tail
 // elements are handled one by one by the first threads of block 0.  Each thread keeps NV
 // packs per array in flight.
@@ -164,6 +179,24 @@ struct DotOp {
   __device__ __forceinline__ static Acc init() { return T(0); }
   __device__ __forceinline__ static void accum(Acc& a, T x, T y, int64_t) { a = x * y + a; }
   __device__ __forceinline__ static void slot_accum(Slot& a, T x, T y, int) { a = x * y + a; }
+  __device__ __forceinline__ static Acc combine(Acc a, Acc b) { return a + b; }
+  __device__ __forceinline__ static Acc shfl(Acc a, int m) { return shfl_xor(a, m); }
+  __device__ __forceinline__ static Out finalize(Acc a) { return a; }
+};
+// dsdot: float inputs, every product and the whole sum in double (a product of two floats is
+// exact in double, so the only rounding is the summation's).
+struct DsdotOp {
+  static constexpr bool kArgmax = false;
+  static constexpr int kPacks = 4;
+  using Acc = double;
+  using Out = double;
+  using Slot = double;
+  __device__ __forceinline__ static Slot slot_init() { return 0.0; }
+  __device__ __forceinline__ static Acc slot_to_acc(Slot s, int64_t, int64_t) { return s; }
+  static constexpr bool RY = true;
+  __device__ __forceinline__ static Acc init() { return 0.0; }
+  __device__ __forceinline__ static void accum(Acc& a, float x, float y, int64_t) { a = (double)x * (double)y + a; }
+  __device__ __forceinline__ static void slot_accum(Slot& a, float x, float y, int) { a = (double)x * (double)y + a; }
   __device__ __forceinline__ static Acc combine(Acc a, Acc b) { return a + b; }
   __device__ __forceinline__ static Acc shfl(Acc a, int m) { return shfl_xor(a, m); }
   __device__ __forceinline__ static Out finalize(Acc a) { return a; }
@@ -459,6 +492,11 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_strided(const T* __restric
   reduce_finish<Op>(r, partials, ticket, result);
 }
 
+// sdsdot's last step: result = (float)(sb + the double-accumulated dot), rounded once.
+__global__ void sdsdot_finish(const double* __restrict__ acc, float sb, float* __restrict__ result) {
+  *result = (float)((double)sb + *acc);
+}
+
 // ------------------------------------------------------------------------------- host side
 static int grid_cap() { return sm_count() * (int)knob(kKnobL1BlocksPerSm); }
 
@@ -575,6 +613,23 @@ using namespace b2;
   if (int e = check_vec(n, x, incx, XP, XP + 1)) return e;     \
   if (int e = check_vec(n, y, incy, XP + 2, XP + 3)) return e;
 
+// rotm: param is a HOST array {flag, h11, h21, h12, h22}; the flag decides which entries are read.
+template <typename T>
+static int rotm_impl(const b2_ctx* ctx, int64_t n, T* x, int64_t incx, T* y, int64_t incy, const T* param) {
+  constexpr int XP = 2;
+  B2_L1_TWO_VEC_CHECK();
+  if (param == nullptr) return -6;
+  const T flag = param[0];
+  RotmOp<T> op;
+  if (flag == T(-1)) op = RotmOp<T>{param[1], param[3], param[2], param[4]};
+  else if (flag == T(0)) op = RotmOp<T>{T(1), param[3], param[2], T(1)};
+  else if (flag == T(1)) op = RotmOp<T>{param[1], T(1), T(-1), param[4]};
+  else if (flag == T(-2)) {  // H = I: nothing to do
+    Launch l;
+    return make_launch(ctx, &l);
+  } else return -6;
+  return run_map<T>(ctx, op, n, x, incx, y, incy);
+}
 extern "C" {
 
 int b2_saxpy(const b2_ctx* ctx, int64_t n, float alpha, const float* x, int64_t incx, float* y, int64_t incy) {
@@ -652,6 +707,36 @@ int b2_ddot(const b2_ctx* ctx, int64_t n, const double* x, int64_t incx, const d
   B2_L1_TWO_VEC_CHECK();
   if (result == nullptr) return -6;
   return run_reduce<double, DotOp<double>>(ctx, n, x, incx, y, incy, result);
+}
+
+int b2_srotm(const b2_ctx* ctx, int64_t n, float* x, int64_t incx, float* y, int64_t incy, const float* param) {
+  return rotm_impl<float>(ctx, n, x, incx, y, incy, param);
+}
+int b2_drotm(const b2_ctx* ctx, int64_t n, double* x, int64_t incx, double* y, int64_t incy, const double* param) {
+  return rotm_impl<double>(ctx, n, x, incx, y, incy, param);
+}
+
+int b2_dsdot(const b2_ctx* ctx, int64_t n, const float* x, int64_t incx, const float* y, int64_t incy,
+             double* result) {
+  constexpr int XP = 2;
+  B2_L1_TWO_VEC_CHECK();
+  if (result == nullptr) return -6;
+  return run_reduce<float, DsdotOp>(ctx, n, x, incx, y, incy, result);
+}
+int b2_sdsdot(const b2_ctx* ctx, int64_t n, float sb, const float* x, int64_t incx, const float* y, int64_t incy,
+              float* result) {
+  constexpr int XP = 3;
+  B2_L1_TWO_VEC_CHECK();
+  if (result == nullptr) return -7;
+  Launch l;
+  if (int st = make_launch(ctx, &l)) return st;
+  // the double sum lands in the workspace, behind the block partials of the reduction
+  const size_t off = ((size_t)grid_cap() * sizeof(double) + 255) / 256 * 256;
+  if (l.scratch_bytes < off + sizeof(double)) return B2_STATUS_WORKSPACE_TOO_SMALL;
+  double* acc = reinterpret_cast<double*>(l.scratch + off);
+  if (int st = run_reduce<float, DsdotOp>(ctx, n, x, incx, y, incy, acc)) return st;
+  sdsdot_finish<<<1, 1, 0, l.stream>>>(acc, sb, result);
+  return check_launch();
 }
 
 #define B2_L1_ONE_VEC_REDUCE(NAME, T, OP, OUT)                                          \
