@@ -240,13 +240,34 @@ class GpuWorkload:
                 events[k][1].record()
 
 
-def next_rows_leg(wl: GpuWorkload, steps: int, peak: float):
-    """The routines beyond the 14 of the headline metric (built after them: syr, syr2), timed the
-    same way (L2 swept, one event bracket per call, median) on a 256 MiB working set; they are NOT
-    part of `value`.  They update the general matrix of the ger variants in place: this leg runs
-    after everything else."""
+def next_rows_leg(wl: GpuWorkload, steps: int, peak: float, only=None):
+    """The routines beyond the 14 of the headline metric (built after them: syr, syr2, rotm, dsdot,
+    sdsdot), timed the same way (L2 swept, one event bracket per call, median) on 256 MiB working
+    sets; they are NOT part of `value`.  syr / syr2 update the general matrix of the ger variants in
+    place and rotm rotates the level-1 vectors: this leg runs after everything else."""
     torch, b2, ctx, B = wl.torch, wl.b2, wl.ctx, wl.buf
     rows = []
+
+    def timed(name, call, touched):
+        if only and not any(k in name for k in only.split(",")):
+            return
+        ts = []
+        for it in range(steps + 3):
+            wl.sweep_l2()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            call()
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                ts.append(e0.elapsed_time(e1))
+        ts.sort()
+        ms = ts[len(ts) // 2]
+        gbs = touched / (ms * 1e-3) / 1e9
+        rows.append({"name": name, "ms": round(ms, 4), "gbs": round(gbs, 1), "frac": round(gbs / peak, 4)})
+
+    dres = torch.zeros(1, dtype=torch.float64, device=wl.dev)
+    sres = torch.zeros(1, dtype=torch.float32, device=wl.dev)
     for dt, s in (("f32", 4), ("f64", 8)):
         if (dt, "ager") not in B:
             continue
@@ -255,27 +276,24 @@ def next_rows_leg(wl: GpuWorkload, steps: int, peak: float):
         for r in ("syr", "syr2"):
             for ul, un in ((UP, "u"), (LO, "l")):
                 for inc in (1, 2):
-                    ts = []
-                    for it in range(steps + 3):
-                        wl.sweep_l2()
-                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                        e0.record()
-                        if r == "syr":
-                            b2.syr(ctx, ROW, ul, n, 1e-3, B[dt, "vx0"], inc, B[dt, "ager"], n)
-                        else:
-                            b2.syr2(ctx, ROW, ul, n, 1e-3, B[dt, "vx0"], inc, B[dt, "vy0"], inc, B[dt, "ager"], n)
-                        e1.record()
-                        torch.cuda.synchronize()
-                        if it >= 3:
-                            ts.append(e0.elapsed_time(e1))
-                    ts.sort()
-                    ms = ts[len(ts) // 2]
+                    if r == "syr":
+                        call = lambda: b2.syr(ctx, ROW, ul, n, 1e-3, B[dt, "vx0"], inc, B[dt, "ager"], n)
+                    else:
+                        call = lambda: b2.syr2(ctx, ROW, ul, n, 1e-3, B[dt, "vx0"], inc, B[dt, "vy0"], inc,
+                                               B[dt, "ager"], n)
                     nvec = 1 if r == "syr" else 2
-                    touched = 2 * tri * s + nvec * n * s * inc
-                    gbs = touched / (ms * 1e-3) / 1e9
-                    rows.append({"name": f"{r}_{un}_{dt}_inc{inc}", "ms": round(ms, 4), "gbs": round(gbs, 1),
-                                 "frac": round(gbs / peak, 4)})
-    return {"note": "rows built after the headline set; bytes = 2 x stored triangle + vectors; not part of `value`",
+                    timed(f"{r}_{un}_{dt}_inc{inc}", call, 2 * tri * s + nvec * n * s * inc)
+        for inc in (1, 2):
+            nv = (128 * MIB // s) // inc  # two vectors, 128 MiB span each
+            x, y = B[dt, "x"], B[dt, "y"]
+            # a plain rotation written as a full H (flag -1): magnitudes stay put over the repeats
+            timed(f"rotm_{dt}_inc{inc}", lambda: b2.rotm(ctx, nv, x, inc, y, inc, [-1.0, 0.6, -0.8, 0.8, 0.6]),
+                  4 * nv * s * inc)
+            if dt == "f32":
+                timed(f"dsdot_inc{inc}", lambda: b2.dsdot(ctx, nv, x, inc, y, inc, dres), 2 * nv * s * inc)
+                timed(f"sdsdot_inc{inc}", lambda: b2.sdsdot(ctx, nv, 0.5, x, inc, y, inc, sres), 2 * nv * s * inc)
+    return {"note": "rows built after the headline set; bytes = touched sectors (2 x stored triangle + vectors for "
+                    "syr/syr2, spans for the level-1 rows); not part of `value`",
             "geomean_frac": geomean([r["frac"] for r in rows]), "variants": rows}
 
 
@@ -465,6 +483,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--filter", default=None, help="only variants whose name contains one of these comma-separated "
                                                    "strings (tuning runs; the headline run uses all)")
+    ap.add_argument("--next-only", action="store_true", help="time only the rows built after the headline set "
+                                                             "(--filter then selects among those)")
     ap.add_argument("--table", default=None, help="also write the per-variant table (JSON) to this path")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -484,6 +504,12 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     from paper_2411_07211_b200 import binding as b2
+    if args.next_only:
+        if world > 1:
+            raise SystemExit("--next-only is a single-GPU profiling aid")
+        wl = GpuWorkload(device, None)
+        print(json.dumps({"next_rows": next_rows_leg(wl, args.steps, peak_gbs()[0], args.filter)}))
+        return
     wl = GpuWorkload(device, args.filter)
     nv = len(wl.specs)
     warm = max(3, args.warmup)
