@@ -292,6 +292,27 @@ def next_rows_leg(wl: GpuWorkload, steps: int, peak: float, only=None):
             if dt == "f32":
                 timed(f"dsdot_inc{inc}", lambda: b2.dsdot(ctx, nv, x, inc, y, inc, dres), 2 * nv * s * inc)
                 timed(f"sdsdot_inc{inc}", lambda: b2.sdsdot(ctx, nv, 0.5, x, inc, y, inc, sres), 2 * nv * s * inc)
+    # narrow matrices (the paper's second level-2 workload, Section 6.2.2: N = 40, static sizes up
+    # to 88 (float) / 44 (double), M a power of 2 or 3), in both storage orders
+    tdt = {"f32": torch.float32, "f64": torch.float64}
+    for dt, s, shapes in (("f32", 4, ((1 << 20, 40), (1 << 20, 88), (3 ** 13, 40))),
+                          ("f64", 8, ((1 << 20, 40), (1 << 20, 44), (3 ** 13, 24)))):
+        if (dt, "ager") not in B or (only and "skinny" not in only):
+            continue
+        amax = max(m * n for m, n in shapes)
+        a = wl.synth.vector_torch(0, 17, amax, tdt[dt], wl.dev)
+        for m, n in shapes:
+            xm, ym = B[dt, "x"], B[dt, "y"]  # length-m vectors
+            xn, yn = B[dt, "vx0"], B[dt, "vy"]  # length-n vectors
+            for order, on, lda in ((ROW, "rm", n), (COL, "cm", m)):
+                tag = f"skinny_{m}x{n}_{on}_{dt}"
+                timed(f"gemv_n_{tag}", lambda: b2.gemv(ctx, order, NOTR, m, n, 1.25, a, lda, xn, 1, 0.5, ym, 1),
+                      (m * n + 2 * m + n) * s)
+                timed(f"gemv_t_{tag}", lambda: b2.gemv(ctx, order, TR, m, n, 1.25, a, lda, xm, 1, 0.5, yn, 1),
+                      (m * n + m + 2 * n) * s)
+                timed(f"ger_{tag}", lambda: b2.ger(ctx, order, m, n, 1e-3, xm, 1, xn, 1, a, lda),
+                      (2 * m * n + m + n) * s)
+        del a
     return {"note": "rows built after the headline set; bytes = touched sectors (2 x stored triangle + vectors for "
                     "syr/syr2, spans for the level-1 rows); not part of `value`",
             "geomean_frac": geomean([r["frac"] for r in rows]), "variants": rows}

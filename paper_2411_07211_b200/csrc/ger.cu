@@ -49,6 +49,27 @@ __global__ void __launch_bounds__(kThreads) ger_kernel(T* __restrict__ a, int64_
           for (int e = 0; e < V; ++e) av[ru][u].v[e] = xv[ru] * yv[u][e] + av[ru][u].v[e];
           st_cs<T, V>(a + rowi[ru] * lda + c0 + (u * LPR + q) * V, av[ru][u]);
         }
+    } else if (V > 1 && (c0 + TC <= cols || (cols - c0) % V == 0)) {
+      // only the matrix edge cuts this tile, on pack boundaries (narrow matrices, short row
+      // bands): the loads still go out together, each under its own row / pack predicate.
+      // (Element-wise tiles, V == 1, stay on the plain path below: single-element streaming
+      // stores to rows that start off a sector boundary measured twice as slow.)
+      const int64_t npk = (min(cols, c0 + TC) - c0) / V;  // packs of this tile that exist
+      P av[RU][CU];
+#pragma unroll
+      for (int ru = 0; ru < RU; ++ru)
+#pragma unroll
+        for (int u = 0; u < CU; ++u)
+          if (rowi[ru] < r_end && u * LPR + q < npk) av[ru][u] = ld_cs<T, V>(a + rowi[ru] * lda + c0 + (u * LPR + q) * V);
+#pragma unroll
+      for (int ru = 0; ru < RU; ++ru)
+#pragma unroll
+        for (int u = 0; u < CU; ++u)
+          if (rowi[ru] < r_end && u * LPR + q < npk) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) av[ru][u].v[e] = xv[ru] * yv[u][e] + av[ru][u].v[e];
+            st_cs<T, V>(a + rowi[ru] * lda + c0 + (u * LPR + q) * V, av[ru][u]);
+          }
     } else {
 #pragma unroll
       for (int ru = 0; ru < RU; ++ru) {

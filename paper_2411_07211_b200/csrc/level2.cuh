@@ -190,9 +190,37 @@ __global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args
               if (K::ROWOUT) rowacc[ru] = av[ru][u].v[e] * xcv[c][u][e] + rowacc[ru];
               if (K::COLOUT) colacc[c][u][e] = av[ru][u].v[e] * xrv[ru] + colacc[c][u][e];
             }
+      } else if (K::TRI == TRI_FULL && (V == 1 || (c1 - c0) % V == 0)) {
+        // gemv: a tile that the matrix edge cuts (fewer rows than RB, or a row that ends on a
+        // pack boundary before the tile does): the loads still go out together, each under its
+        // own row / pack predicate.  Narrow matrices (fewer columns than one tile) and short
+        // ones (fewer rows than one step) live entirely here.  A masked pack is zero and meets
+        // a zero x value, so it adds nothing.
+        const int npk = (int)(c1 - c0) / V;  // packs of this tile that exist
+        P av[RU][CU];
+        const T* at = a_rb + c0;
+#pragma unroll
+        for (int ru = 0; ru < RU; ++ru) {
+          const bool rok = lrow0 + ru * kWarps * G < nr;
+#pragma unroll
+          for (int u = 0; u < CU; ++u) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) av[ru][u].v[e] = T(0);
+            if (rok && u * LPR + q < npk) av[ru][u] = ld_nc<T, V>(at + ru * rstride + u * (LPR * V));
+          }
+        }
+#pragma unroll
+        for (int ru = 0; ru < RU; ++ru)
+#pragma unroll
+          for (int u = 0; u < CU; ++u)
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+              if (K::ROWOUT) rowacc[ru] = av[ru][u].v[e] * xcv[c][u][e] + rowacc[ru];
+              if (K::COLOUT) colacc[c][u][e] = av[ru][u].v[e] * xrv[ru] + colacc[c][u][e];
+            }
       } else {
-        // Edge and diagonal tiles: local 32-bit indices; d = (first column) - (first row), so
-        // element (li, lj) lies on the diagonal when d + lj == li.
+        // Diagonal tiles and column edges inside a pack: local 32-bit indices; d = (first column)
+        // - (first row), so element (li, lj) lies on the diagonal when d + lj == li.
         const int64_t d64 = c0 - rb;
         const int d = (int)(d64 > (1 << 24) ? (1 << 24) : d64 < -(1 << 24) ? -(1 << 24) : d64);
         const int nc = (int)(c1 - c0);

@@ -39,7 +39,9 @@ def matbuf(seed, major, minor, lda, dtype):
 
 
 GEMV_SHAPES = [(1, 1), (3, 5), (17, 33), (64, 64), (100, 700), (700, 100), (257, 1031), (1500, 40), (40, 3000),
-               (2049, 513), (130, 2100), (4100, 24)]
+               (2049, 513), (130, 2100), (4100, 24),
+               # narrow shapes of the paper's skinny study (Section 6.2.2): N = 40, N <= 88 / 44, M a power of 2 or 3
+               (2187, 40), (2187, 44), (4096, 88), (88, 4096), (44, 2187), (6561, 8)]
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
