@@ -2,6 +2,7 @@
 // Row-major N is the row-dot kind, row-major T the column-sum kind; a column-major call is
 // the transposed row-major problem (A^T stored row-major), so N and T swap kinds.
 #include "level2.cuh"
+#include "skinny.cuh"
 
 namespace b2 {
 
@@ -41,6 +42,8 @@ static int gemv_impl(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t
   if (rowdot) {
     args.xc = vec_base(x, lenx, incx);
     args.incxc = incx;
+    if (skinny_applies(a, lda, args.rows, args.cols, true))
+      return skinny_rowdot<T>(l, a, args.rows, args.cols, args.xc, incx, alpha, beta, args.y, incy);
     return l2_dispatch<T, GemvRow, true>(l, args, plan_rowout(args, true), true);
   }
   args.xr = vec_base(x, lenx, incx);

@@ -2,6 +2,7 @@
 // the gemv schedule).  Pure streaming read-modify-write of A: each lane keeps alpha*y_j for
 // its columns in registers and reuses them down a band of rows, x_i is a broadcast load.
 #include "level2.cuh"
+#include "skinny.cuh"
 
 namespace b2 {
 
@@ -141,6 +142,7 @@ static int ger_impl(const b2_ctx* ctx, int order, int64_t m, int64_t n, T alpha,
   const T* yc = rm ? vec_base(y, n, incy) : vec_base(x, m, incx);
   const int64_t incyc = rm ? incy : incx;
   constexpr int V = VecLen<T>::value;
+  if (skinny_applies(a, lda, rows, cols, false)) return skinny_ger<T>(l, a, rows, cols, xr, incxr, yc, incyc, alpha);
   if (aligned_to(a, 16) && lda % V == 0) return ger_shape<T, V>(l, a, lda, rows, cols, xr, incxr, yc, incyc, alpha);
   return ger_shape<T, 1>(l, a, lda, rows, cols, xr, incxr, yc, incyc, alpha);
 }

@@ -1,0 +1,183 @@
+// Narrow-matrix kernels for gemv (row-dot kind) and ger (Section 6.2.2 of the paper: a separate
+// schedule for matrices whose row is a few vector registers long, with the reused vector staged
+// once and static sizes up to 88 floats / 44 doubles).
+//
+// Setting: the canonical row-major view has many rows and a row of PPR 16-byte packs, PPR <= 22,
+// stored without padding (lda == cols), so the whole matrix is ONE contiguous stream of packs and
+// a pack never straddles two rows.  The general tile kernel gives each row its own group of 8,
+// 16 or 32 lanes; at 10 or 11 packs per row a third of the lanes idle.  Here a warp instead takes
+// "chunks" of 32 rows = 32 * PPR consecutive packs and reads them with PPR fully coalesced
+// instructions: lane l, instruction k holds pack k*32 + l of the chunk, which belongs to row
+// (k*32 + l) / PPR and column pack (k*32 + l) % PPR.  Neither quotient is computed by a division:
+// both advance by fixed steps from one instruction to the next.
+//   row-dot: each pack is multiplied with its slice of x (shared memory) into one partial, the
+//            partials go to shared memory in stream order, and lane l then adds the PPR
+//            partials of row l -- a segmented sum without any cross-lane traffic.
+//   ger:     lane l holds alpha * x of row l of the chunk; a pack gets its row's value by a
+//            shuffle and its slice of y from shared memory.
+#pragma once
+
+#include "common.cuh"
+
+namespace b2 {
+
+constexpr int kSkinnyMaxPpr = 22;       // 88 floats / 44 doubles per row
+constexpr int kSkinnyGroup = 11;        // packs of a lane in flight together: a chunk is one or two groups
+constexpr int64_t kSkinnyMinRows = 2048;
+
+// True when the flat-stream kernels apply and pay: few packs per row, no padding, aligned base,
+// and a row length that leaves more than 30 % of the lanes idle in the general kernel (which
+// gives a row 8, 16 or 32 lanes).  Measured on 2^20-row matrices: at 10 and 22 packs per row the
+// flat kernels win (float row-dot 0.71 -> 0.80 and 0.87 -> 0.92 of the copy rate, ger 0.72 ->
+// 0.83), at 12 packs (75 % of the lanes busy) they lose.  The double row-dot is slower flat at
+// every width measured (0.51 against 0.63): it stays on the general kernel.
+template <typename T>
+static bool skinny_applies(const T* a, int64_t lda, int64_t rows, int64_t cols, bool rowdot) {
+  constexpr int V = VecLen<T>::value;
+  if (rowdot && sizeof(T) == 8) return false;
+  if (rows < kSkinnyMinRows || cols != lda || cols % V != 0 || !aligned_to(a, 16)) return false;
+  const int64_t ppr = cols / V;
+  if (ppr < 1 || ppr > kSkinnyMaxPpr) return false;
+  const int64_t lanes = ppr <= 8 ? 8 : ppr <= 16 ? 16 : 32;
+  return 10 * ppr < 7 * lanes;
+}
+
+// y_i <- alpha * sum_j a_ij x_j + beta * y_i over a flat pack stream.  x, y: vec_base() bases.
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 3) skinny_rowdot_kernel(const T* __restrict__ a, int64_t rows, int ppr,
+                                                                    const T* __restrict__ x, int64_t incx, T alpha,
+                                                                    T beta, T* __restrict__ y, int64_t incy,
+                                                                    int64_t nchunks) {
+  constexpr int V = VecLen<T>::value;
+  using P = Pack<T, V>;
+  __shared__ __align__(16) T xs[kSkinnyMaxPpr * V];
+  __shared__ T part[kWarps][(kSkinnyMaxPpr + 1) * 32];  // row r at r * (ppr | 1): an odd pitch spreads the banks
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int t = threadIdx.x; t < ppr * V; t += kThreads) xs[t] = __ldg(x + t * incx);
+  __syncthreads();
+  const int cstep = 32 % ppr, rstep = 32 / ppr;  // per instruction: column pack += cstep (mod ppr), row += rstep (+ carry)
+  const int c_first = lane % ppr, r_first = lane / ppr;
+  const int pitch = ppr | 1;
+  for (int64_t chunk = (int64_t)blockIdx.x * kWarps + warp; chunk < nchunks; chunk += (int64_t)gridDim.x * kWarps) {
+    const int64_t row0 = chunk * 32;
+    const int nrows = (int)min((int64_t)32, rows - row0);
+    const int npacks = nrows * ppr;  // packs of this chunk that exist
+    const P* src = reinterpret_cast<const P*>(a) + row0 * ppr;
+    int c = c_first, r = r_first;
+    for (int k0 = 0; k0 < ppr; k0 += kSkinnyGroup) {
+      P av[kSkinnyGroup];
+#pragma unroll
+      for (int g = 0; g < kSkinnyGroup; ++g) {
+        const int pos = (k0 + g) * 32 + lane;
+        if (k0 + g < ppr && pos < npacks) av[g] = ld_nc<T, V>(reinterpret_cast<const T*>(src + pos));
+      }
+#pragma unroll
+      for (int g = 0; g < kSkinnyGroup; ++g) {
+        const int pos = (k0 + g) * 32 + lane;
+        if (k0 + g < ppr) {
+          T s = T(0);
+          if (pos < npacks) {
+            const P xv = *reinterpret_cast<const P*>(&xs[c * V]);
+#pragma unroll
+            for (int e = 0; e < V; ++e) s = av[g].v[e] * xv.v[e] + s;
+          }
+          part[warp][r * pitch + c] = s;
+          c += cstep;
+          r += rstep;
+          if (c >= ppr) {
+            c -= ppr;
+            r += 1;
+          }
+        }
+      }
+    }
+    __syncwarp();
+    if (lane < nrows) {
+      T s = T(0);
+      for (int k = 0; k < ppr; ++k) s += part[warp][lane * pitch + k];
+      T* yp = y + (row0 + lane) * incy;
+      *yp = beta != T(0) ? alpha * s + beta * *yp : alpha * s;
+    }
+    __syncwarp();  // part is rewritten by the next chunk
+  }
+}
+
+// a_ij <- alpha * x_i * y_j + a_ij over a flat pack stream.  xr indexed by row, yc by column.
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 3) skinny_ger_kernel(T* __restrict__ a, int64_t rows, int ppr,
+                                                                 const T* __restrict__ xr, int64_t incxr,
+                                                                 const T* __restrict__ yc, int64_t incyc, T alpha,
+                                                                 int64_t nchunks) {
+  constexpr int V = VecLen<T>::value;
+  using P = Pack<T, V>;
+  __shared__ __align__(16) T ys[kSkinnyMaxPpr * V];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int t = threadIdx.x; t < ppr * V; t += kThreads) ys[t] = __ldg(yc + t * incyc);
+  __syncthreads();
+  const int cstep = 32 % ppr, rstep = 32 / ppr;  // per instruction: column pack += cstep (mod ppr), row += rstep (+ carry)
+  const int c_first = lane % ppr, r_first = lane / ppr;
+  for (int64_t chunk = (int64_t)blockIdx.x * kWarps + warp; chunk < nchunks; chunk += (int64_t)gridDim.x * kWarps) {
+    const int64_t row0 = chunk * 32;
+    const int nrows = (int)min((int64_t)32, rows - row0);
+    const int npacks = nrows * ppr;
+    P* dst = reinterpret_cast<P*>(a) + row0 * ppr;
+    const T xrow = lane < nrows ? alpha * __ldg(xr + (row0 + lane) * incxr) : T(0);
+    int c = c_first, r = r_first;
+    for (int k0 = 0; k0 < ppr; k0 += kSkinnyGroup) {
+      P av[kSkinnyGroup];
+#pragma unroll
+      for (int g = 0; g < kSkinnyGroup; ++g) {
+        const int pos = (k0 + g) * 32 + lane;
+        if (k0 + g < ppr && pos < npacks) av[g] = ld_cs<T, V>(reinterpret_cast<const T*>(dst + pos));
+      }
+#pragma unroll
+      for (int g = 0; g < kSkinnyGroup; ++g) {
+        const int pos = (k0 + g) * 32 + lane;
+        if (k0 + g < ppr) {  // uniform over the warp: the shuffle below is executed by all lanes
+          const T xi = __shfl_sync(0xffffffffu, xrow, r & 31);
+          if (pos < npacks) {
+            const P yv = *reinterpret_cast<const P*>(&ys[c * V]);
+#pragma unroll
+            for (int e = 0; e < V; ++e) av[g].v[e] = xi * yv.v[e] + av[g].v[e];
+            st_cs<T, V>(reinterpret_cast<T*>(dst + pos), av[g]);
+          }
+          c += cstep;
+          r += rstep;
+          if (c >= ppr) {
+            c -= ppr;
+            r += 1;
+          }
+        }
+      }
+    }
+  }
+}
+
+template <typename T>
+static int skinny_grid(int64_t nchunks) {
+  const int64_t blocks = (nchunks + kWarps - 1) / kWarps;
+  const int64_t cap = (int64_t)sm_count() * 3;  // one resident wave (three blocks per SM)
+  return (int)(blocks < cap ? blocks : cap);
+}
+
+template <typename T>
+static int skinny_rowdot(const Launch& l, const T* a, int64_t rows, int64_t cols, const T* x, int64_t incx, T alpha,
+                         T beta, T* y, int64_t incy) {
+  const int ppr = (int)(cols / VecLen<T>::value);
+  const int64_t nchunks = (rows + 31) / 32;
+  skinny_rowdot_kernel<T><<<skinny_grid<T>(nchunks), kThreads, 0, l.stream>>>(a, rows, ppr, x, incx, alpha, beta, y,
+                                                                             incy, nchunks);
+  return check_launch();
+}
+
+template <typename T>
+static int skinny_ger(const Launch& l, T* a, int64_t rows, int64_t cols, const T* xr, int64_t incxr, const T* yc,
+                      int64_t incyc, T alpha) {
+  const int ppr = (int)(cols / VecLen<T>::value);
+  const int64_t nchunks = (rows + 31) / 32;
+  skinny_ger_kernel<T><<<skinny_grid<T>(nchunks), kThreads, 0, l.stream>>>(a, rows, ppr, xr, incxr, yc, incyc, alpha,
+                                                                          nchunks);
+  return check_launch();
+}
+
+}  // namespace b2
