@@ -48,6 +48,26 @@ static int gemv_impl(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t
   }
   args.xr = vec_base(x, lenx, incx);
   args.incxr = incx;
+  if (skinny_colsum_applies(a, lda, args.rows, args.cols)) {
+    const int ppr = (int)(args.cols / VecLen<T>::value);
+    const int64_t rows_per_step = (int64_t)(32 / ppr) * kColsumGroup;
+    const int64_t nsteps = (args.rows + rows_per_step - 1) / rows_per_step;
+    const int64_t want = (nsteps + kWarps - 1) / kWarps, cap = (int64_t)sm_count() * 4;
+    const int grid = (int)(want < cap ? want : cap);
+    if ((size_t)grid * args.cols * sizeof(T) <= l.scratch_bytes) {
+      args.colpart = reinterpret_cast<T*>(l.scratch);
+      args.nrs = grid;  // one partial row per block; the finalize kernel adds all of them
+      args.ncs = 1;
+      args.nct = 1;
+      args.ctiles_per_cta = 1;
+      args.rows_per_cta = args.rows;
+      args.direct = 0;
+      skinny_colsum_kernel<T><<<grid, kThreads, 0, l.stream>>>(a, args.rows, ppr, args.xr, incx, args.colpart, nsteps);
+      if (int st = check_launch()) return st;
+      launch_finalize<T, GemvCol, 32>(l, args, 1, (int)args.cols, args.cols);
+      return check_launch();
+    }
+  }
   return l2_dispatch<T, GemvCol, true>(l, args, plan_colout(args, true, knob(kKnobGemvTRows)), true);
 }
 

@@ -153,6 +153,79 @@ __global__ void __launch_bounds__(kThreads, 3) skinny_ger_kernel(T* __restrict__
   }
 }
 
+// Column sums of a narrow matrix (the gemv kind whose output has one entry per column):
+// colpart[block][j] = sum over the block's rows of a_ij * x_i.  A lane's column must not change
+// from load to load (its sums live in registers), so here a row gets exactly PPR lanes: a warp
+// instruction covers G = 32 / PPR whole rows with its first G * PPR lanes -- 30 of 32 lanes at 10
+// packs per row, where power-of-two row groups would use 20.  The loads of one instruction are
+// still one contiguous run of packs.  Each block leaves one partial row; the general finalize
+// kernel adds the partials in a fixed order and applies alpha / beta.
+constexpr int kColsumGroup = 8;  // instructions of a lane in flight together
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 4) skinny_colsum_kernel(const T* __restrict__ a, int64_t rows, int ppr,
+                                                                    const T* __restrict__ xr, int64_t incxr,
+                                                                    T* __restrict__ colpart, int64_t nsteps) {
+  constexpr int V = VecLen<T>::value;
+  using P = Pack<T, V>;
+  __shared__ T sm[kWarps][32 * V];
+  grid_dep_launch();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = 32 / ppr;
+  const bool active = lane < G * ppr;
+  const int g = lane / ppr;  // row of this lane inside an instruction (valid when active)
+  const int64_t rows_per_step = (int64_t)G * kColsumGroup;
+  T acc[V];
+#pragma unroll
+  for (int e = 0; e < V; ++e) acc[e] = T(0);
+  for (int64_t step = (int64_t)blockIdx.x * kWarps + warp; step < nsteps; step += (int64_t)gridDim.x * kWarps) {
+    const int64_t row0 = step * rows_per_step;
+    const P* src = reinterpret_cast<const P*>(a) + row0 * ppr + lane;
+    P av[kColsumGroup];
+    T xv[kColsumGroup];
+#pragma unroll
+    for (int k = 0; k < kColsumGroup; ++k) {
+      const int64_t row = row0 + k * G + g;
+      const bool ok = active && row < rows;
+      xv[k] = T(0);
+#pragma unroll
+      for (int e = 0; e < V; ++e) av[k].v[e] = T(0);
+      if (ok) {
+        av[k] = ld_nc<T, V>(reinterpret_cast<const T*>(src + (int64_t)k * G * ppr));
+        xv[k] = __ldg(xr + row * incxr);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < kColsumGroup; ++k)
+#pragma unroll
+      for (int e = 0; e < V; ++e) acc[e] = av[k].v[e] * xv[k] + acc[e];
+  }
+  // lanes g * ppr + q (all g, all warps) hold partial sums of column pack q
+#pragma unroll
+  for (int e = 0; e < V; ++e) sm[warp][lane * V + e] = active ? acc[e] : T(0);
+  __syncthreads();
+  for (int j = threadIdx.x; j < ppr * V; j += kThreads) {
+    const int q = j / V, e = j % V;
+    T s = T(0);
+    for (int w = 0; w < kWarps; ++w)
+      for (int gg = 0; gg < G; ++gg) s += sm[w][(gg * ppr + q) * V + e];
+    colpart[(int64_t)blockIdx.x * (ppr * V) + j] = s;
+  }
+}
+
+// Exact-width row groups pay when they keep clearly more lanes busy than the general kernel's
+// power-of-two groups (a margin of 15 % of the warp).
+template <typename T>
+static bool skinny_colsum_applies(const T* a, int64_t lda, int64_t rows, int64_t cols) {
+  constexpr int V = VecLen<T>::value;
+  if (rows < kSkinnyMinRows || cols != lda || cols % V != 0 || !aligned_to(a, 16)) return false;
+  const int64_t ppr = cols / V;
+  if (ppr < 1 || ppr > 16) return false;
+  const int64_t lanes = ppr <= 8 ? 8 : 16;          // the general kernel's row group
+  const int64_t busy = (32 / ppr) * ppr;            // lanes busy here, of 32
+  return 100 * busy >= 100 * 32 * ppr / lanes + 15 * 32;
+}
+
 template <typename T>
 static int skinny_grid(int64_t nchunks) {
   const int64_t blocks = (nchunks + kWarps - 1) / kWarps;
