@@ -47,7 +47,9 @@ def dvec(seed, stream, n, dtype, inc=1):
 
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float64])
-@pytest.mark.parametrize("m,n", [(4096, 4096), (8192, 8192), (5760, 5760), (16384, 16384), (1 << 20, 64), (64, 1 << 20)])
+@pytest.mark.parametrize("m,n", [(4096, 4096), (8192, 8192), (5760, 5760), (16384, 16384), (1 << 20, 64), (64, 1 << 20),
+                                 # the narrow shapes the bench's next-rows leg times (flat-stream kernels)
+                                 (1 << 20, 40), (1 << 20, 88), (1 << 20, 44), (3 ** 13, 40), (3 ** 13, 24)])
 def test_gemv_ger_config_sizes(b2, ctx, dtype, m, n):
     seed = 31
     a = synth.matrix_torch(seed, 1, m, n, n, TD[dtype], "cuda")
