@@ -13,8 +13,8 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobTrsvDebugSkip   */ -1,
     /* kKnobTriWide         */ 0,
     /* kKnobTrsvPrefetchBytes */ 48 << 20,
-    /* kKnobTrsvFront       */ 1,
-    /* kKnobTrsvCluster     */ 1,
+    /* kKnobTrsvFront       */ 2,
+    /* kKnobTrsvCluster     */ 0,
 };
 
 unsigned long long g_launch_count = 0;

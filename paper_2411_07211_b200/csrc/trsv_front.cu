@@ -247,8 +247,9 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
   T* xs = Ms + (PM ? NB * SP : 0);              // [2][NB] x values of the current / next tile
   T* rbuf = xs + 2 * NB;                        // r = b - sum, the vector of the final trip
   T* bvec = rbuf + NB;
+  T* red = bvec + NB;                           // [kT / 32][NB] per-warp partial row sums (column-type views)
   // x of the earlier rows of this cluster: [CS][NB * WPE] words {payload, row + 1}, written by their blocks
-  unsigned long long* xrecv = reinterpret_cast<unsigned long long*>(bvec + NB);
+  unsigned long long* xrecv = reinterpret_cast<unsigned long long*>(red + (kT / 32) * NB);
   __shared__ unsigned s_ticket[2];
 #ifdef B2_TRSV_TRACE
   __shared__ unsigned long long s_trace[16];
@@ -256,9 +257,17 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
 
   const int ct = (int)threadIdx.x, warp = ct >> 5, lane = ct & 31;
   const int rg = ct >> 4, cg = ct & 15;
-  // the row (solve order inside the block) this thread may own: sub-block row a = cg / LPO
-  const int ti = ((cg / LPO) / V) * H + V * rg + ((cg / LPO) % V);
-  const bool owner = (cg % LPO) == 0;
+  // Row-type views: a 16 x 16 thread grid, thread (rg, cg) holds an RS x RS sub-block and the row
+  // sums run over the 16 lanes that share rg.  Column-type views (a tile of op(A) is the transpose
+  // of a stored tile): lanes must run along the STORED rows or a load instruction touches 16 rows
+  // for one sector each, so lane l holds rows V*l .. V*l+V-1 of op(A), warp w the columns
+  // w*JT .. w*JT+JT-1 (JT stored rows, each read as one 512-byte run by the warp), and the row
+  // sums run across the warps through `red`.
+  constexpr int JT = NB / (kT / 32);
+  static_assert(JT * V == E, "both layouts hold the same number of elements per thread");
+  // the row (solve order inside the block) this thread may own
+  const int ti = COLTYPE ? (ct & (NB - 1)) : ((cg / LPO) / V) * H + V * rg + ((cg / LPO) % V);
+  const bool owner = COLTYPE ? ct < NB : (cg % LPO) == 0;
 
   Waiter wt;
   wt.budget = p.wait_limit ? p.wait_limit : (1ull << 22);
@@ -325,17 +334,14 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
           }
         }
       } else {
+        // m[jj * V + e] = op(A)(row V*lane + e, column warp*JT + jj) = stored (c0 + column, rr0 + row')
+        const int m0 = BACKWARD ? NB - V * lane - V : V * lane;  // ascending memory run of the pack
 #pragma unroll
-        for (int b = 0; b < RS; ++b) {
-          const int j = (b / V) * H + V * cg + (b % V);
-          const T* src = base + (c0 + j) * ld + rr0;
+        for (int jj = 0; jj < JT; ++jj) {
+          const T* src = base + (c0 + warp * JT + jj) * ld + rr0 + m0;
+          const P pk = smem ? *reinterpret_cast<const P*>(src) : ld_nc<T, V>(src);
 #pragma unroll
-          for (int ha = 0; ha < RS / V; ++ha) {
-            const int m0 = BACKWARD ? NB - ha * H - V * rg - V : ha * H + V * rg;  // ascending memory run of the chunk
-            const P pk = smem ? *reinterpret_cast<const P*>(src + m0) : ld_nc<T, V>(src + m0);
-#pragma unroll
-            for (int e = 0; e < V; ++e) m[(ha * V + (BACKWARD ? V - 1 - e : e)) * RS + b] = pk.v[e];
-          }
+          for (int e = 0; e < V; ++e) m[jj * V + (BACKWARD ? V - 1 - e : e)] = pk.v[e];
         }
       }
     };
@@ -349,7 +355,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
         fill(m, s == yt ? Wt : Ms, SP, 0, 0, true);
       } else if (nbI == NB && nbJ == NB) {
         fill(m, p.a, p.lda, c0, r0, false);
-      } else {
+      } else if (!COLTYPE) {
 #pragma unroll
         for (int a = 0; a < RS; ++a)
 #pragma unroll
@@ -357,7 +363,17 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
             const int i = (a / V) * H + V * rg + (a % V), jc = (b / V) * H + V * cg + (b % V);
             const bool ok = i < nbI && jc < nbJ;
             const int64_t mrow = r0 + (ok ? sidx(i) : 0), mcol = c0 + jc;
-            m[a * RS + b] = ok ? __ldg(COLTYPE ? p.a + mcol * p.lda + mrow : p.a + mrow * p.lda + mcol) : T(0);
+            m[a * RS + b] = ok ? __ldg(p.a + mrow * p.lda + mcol) : T(0);
+          }
+      } else {
+#pragma unroll
+        for (int jj = 0; jj < JT; ++jj)
+#pragma unroll
+          for (int e = 0; e < V; ++e) {
+            const int i = V * lane + e, jc = warp * JT + jj;
+            const bool ok = i < nbI && jc < nbJ;
+            const int64_t mrow = r0 + (ok ? sidx(i) : 0), mcol = c0 + jc;
+            m[jj * V + e] = ok ? __ldg(p.a + mcol * p.lda + mrow) : T(0);
           }
       }
     };
@@ -535,15 +551,22 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       {  // the tile, rows in solve order, through registers into Ms
         T t1[E];
         load_tile(t1, k - 1, true);
+        if (!COLTYPE) {
 #pragma unroll
-        for (int a = 0; a < RS; ++a)
+          for (int a = 0; a < RS; ++a)
 #pragma unroll
-          for (int hb = 0; hb < RS / V; ++hb) {
-            P pk;
+            for (int hb = 0; hb < RS / V; ++hb) {
+              P pk;
 #pragma unroll
-            for (int e = 0; e < V; ++e) pk.v[e] = t1[a * RS + hb * V + e];
-            *reinterpret_cast<P*>(Ms + ((a / V) * H + V * rg + (a % V)) * SP + hb * H + V * cg) = pk;
-          }
+              for (int e = 0; e < V; ++e) pk.v[e] = t1[a * RS + hb * V + e];
+              *reinterpret_cast<P*>(Ms + ((a / V) * H + V * rg + (a % V)) * SP + hb * H + V * cg) = pk;
+            }
+        } else {
+#pragma unroll
+          for (int jj = 0; jj < JT; ++jj)
+#pragma unroll
+            for (int e = 0; e < V; ++e) Ms[(V * lane + e) * SP + warp * JT + jj] = t1[jj * V + e];
+        }
       }
       bar_sync(kBar, kT);
       constexpr int JW = NB * NB / (4 * kT);  // columns per thread: 16 (float) / 4 (double), 4 rows
@@ -666,20 +689,42 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       B2_CTRACE(ct == 0 && srow == k - 1 && !is_y, 8);
       B2_CTRACE(ct == 0 && it == k / 2, 14);  // barrier passed
       const T* vec = is_y ? rbuf : xbuf_s;
-      T xv[RS], part[RS];
+      T s;
+      if constexpr (!COLTYPE) {
+        T xv[RS], part[RS];
 #pragma unroll
-      for (int hb = 0; hb < RS / V; ++hb) {
-        const P pk = *reinterpret_cast<const P*>(vec + hb * H + V * cg);
+        for (int hb = 0; hb < RS / V; ++hb) {
+          const P pk = *reinterpret_cast<const P*>(vec + hb * H + V * cg);
 #pragma unroll
-        for (int e = 0; e < V; ++e) xv[hb * V + e] = pk.v[e];
+          for (int e = 0; e < V; ++e) xv[hb * V + e] = pk.v[e];
+        }
+#pragma unroll
+        for (int a = 0; a < RS; ++a) {
+          part[a] = T(0);
+#pragma unroll
+          for (int bcol = 0; bcol < RS; ++bcol) part[a] = cur[a * RS + bcol] * xv[bcol] + part[a];
+        }
+        s = multi_group_sum<16, RS>(part, lane);
+      } else {
+        P part;
+#pragma unroll
+        for (int e = 0; e < V; ++e) part.v[e] = T(0);
+#pragma unroll
+        for (int q = 0; q < JT / V; ++q) {
+          const P pk = *reinterpret_cast<const P*>(vec + warp * JT + q * V);  // the warp's columns: a broadcast
+#pragma unroll
+          for (int u = 0; u < V; ++u)
+#pragma unroll
+            for (int e = 0; e < V; ++e) part.v[e] = cur[(q * V + u) * V + e] * pk.v[u] + part.v[e];
+        }
+        *reinterpret_cast<P*>(red + warp * NB + V * lane) = part;
+        bar_sync(kBar, kT);  // (the next trip writes red only after its own first barrier)
+        s = T(0);
+        if (ct < NB) {
+#pragma unroll
+          for (int w = 0; w < kT / 32; ++w) s += red[w * NB + ct];
+        }
       }
-#pragma unroll
-      for (int a = 0; a < RS; ++a) {
-        part[a] = T(0);
-#pragma unroll
-        for (int bcol = 0; bcol < RS; ++bcol) part[a] = cur[a * RS + bcol] * xv[bcol] + part[a];
-      }
-      const T s = multi_group_sum<16, RS>(part, lane);
       B2_CTRACE(ct == 0 && srow == k - 1 && !is_y, 7);
       B2_CTRACE(ct == 0 && it == k / 2, 15);  // reduced
       const T out = is_m ? yreg - s : s;
@@ -735,7 +780,7 @@ template <typename T>
 constexpr size_t front_smem_bytes(int cs) {
   constexpr int NB = Geo<T>::NB;
   constexpr int SP = NB + 16 / (int)sizeof(T);
-  return sizeof(T) * (size_t)((cs > 1 ? 1 : 2) * NB * SP + (NB / 2) * (NB / 2 + 4) + 4 * NB) +
+  return sizeof(T) * (size_t)((cs > 1 ? 1 : 2) * NB * SP + (NB / 2) * (NB / 2 + 4) + (4 + kT / 32) * NB) +
          (cs > 1 ? (size_t)cs * NB * Words<T>::N * 8 : 0);
 }
 
@@ -801,8 +846,7 @@ int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int6
   constexpr int NB = Geo<T>::NB, V = Geo<T>::V, WPE = Words<T>::N;
   *handled = false;
   if (!knob(kKnobTrsvFront)) return B2_STATUS_OK;
-  // Column-type views (op(A)'s rows strided in memory) load their sub-blocks from 16 memory rows
-  // per request; the block-row kernel is faster there.
+  // (knob value 1 keeps column-type views on the block-row kernel)
   if (coltype && knob(kKnobTrsvFront) < 2) return B2_STATUS_OK;
   if (!aligned_to(a, 16) || lda % V != 0) return B2_STATUS_OK;
   const int64_t nb64 = (n + NB - 1) / NB;
@@ -833,8 +877,9 @@ int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int6
   args.trace = reinterpret_cast<unsigned long long*>(l.scratch + l.scratch_bytes - ((size_t)16 << 20));
 #endif
   *handled = true;
-  // (measured: clusters pay for float; for double, with twice the words per value to push to
-  // seven peers, they do not)
+  // (measured at n = 11520 / 8192: block by block with the premultiplied last tile is the
+  // fastest form for both precisions -- float 156-162 us against 168-175 us in clusters of 8,
+  // double 180 us against 216 us -- so clusters are off by default)
   const bool want_cluster = nb >= 2 && (knob(kKnobTrsvCluster) >= 2 || (knob(kKnobTrsvCluster) == 1 && sizeof(T) == 4));
   if (coltype)
     return backward ? launch_diag<T, true, true>(l, args, nb, want_cluster, unit)
