@@ -31,9 +31,8 @@ FALLBACK_PEAK_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of each kernel template at the bench
 # sizes, from the ncu captures summarised in profiles/kernels_config5_ncu_full.md (same kernels).
 # Set an entry to None when its kernel changes and the counters have not been retaken.
-# trsv: mean of the block-row kernel (271.4 MB) and the sub-block kernel (288.3 MB float, 289.0 MB
-# double), which each serve half of the trsv variants.
-NCU_DRAM_BYTES_PER_LAUNCH = {"trsv": 280.0e6, "l2_tile": 271.3e6, "l1_reduce": 272.3e6, "l1_map": 351.8e6,
+# trsv: the sub-block kernel, which serves every bench variant (273.4-274.0 MB float, 275.3 MB double).
+NCU_DRAM_BYTES_PER_LAUNCH = {"trsv": 274.0e6, "l2_tile": 271.3e6, "l1_reduce": 272.3e6, "l1_map": 351.8e6,
                              "ger": 479.3e6}
 
 
