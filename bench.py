@@ -444,7 +444,7 @@ def oracle_pass(scale: int, seed: int = 0):
 
 def reference_arm(args):
     """`--impl reference`: the oracle, as it stands, on the host cores; each step is one pass over
-    every variant at 1/64 of the bench's element counts (bounded so the run ends in minutes)."""
+    every variant at 1/16 of the bench's element counts (bounded so the run ends in minutes)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -460,12 +460,13 @@ def reference_arm(args):
     value = geomean(per)
     sample = f"every variant at 1/{scale} of the bench element counts (16 MiB working sets), 1 thread"
     print(json.dumps({
-        "impl": "reference", "metric": "achieved GB/s per BLAS-1/2 variant, geomean over variants",
+        "impl": "reference", "metric": "achieved HBM GB/s per BLAS-1/2 variant, geomean over variants",
         "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": wall / max(1, args.steps) * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32+f64", "data": "synthetic",
-        "config": {"workload": "config 5 cross-product (routines x f32/f64 x options x inc 1/2), CPU sample",
-                   "variants": len(per)},
+        "config": {"workload": "config 5: every routine x {f32,f64} x trans/uplo/diag x inc {1,2}, 256 MiB working "
+                               "set per variant, row-major", "variants": len(per), "sample": sample,
+                   "bytes": "touched sectors (span bytes)", "parallelism": "one host core"},
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
