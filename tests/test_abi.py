@@ -58,6 +58,22 @@ def test_argument_validation_without_gpu(b2):
     assert h.b2_strmv(c, b2.ROW_MAJOR, b2.UPPER, b2.NO_TRANS, 0, 2, p, 2, p, 1) == -4
     assert h.b2_dtrsv(c, b2.ROW_MAJOR, b2.UPPER, b2.NO_TRANS, b2.UNIT, 2, p, 1, p, 1) == -7
     assert h.b2_dtrsv(c, b2.ROW_MAJOR, b2.UPPER, b2.NO_TRANS, b2.UNIT, 2, p, 2, p, 0) == -9
+    # the routines built after the headline set
+    assert h.b2_ssyr(c, 7, b2.UPPER, 2, 1.0, p, 1, p, 2) == -1
+    assert h.b2_ssyr(c, b2.ROW_MAJOR, 7, 2, 1.0, p, 1, p, 2) == -2
+    assert h.b2_dsyr(c, b2.ROW_MAJOR, b2.UPPER, 2, 1.0, p, 0, p, 2) == -6
+    assert h.b2_dsyr(c, b2.ROW_MAJOR, b2.UPPER, 2, 1.0, p, 1, p, 1) == -8
+    assert h.b2_ssyr2(c, b2.ROW_MAJOR, b2.UPPER, 2, 1.0, p, 1, None, 1, p, 2) == -7
+    assert h.b2_ssyr2(c, b2.ROW_MAJOR, b2.UPPER, 2, 1.0, p, 1, p, 1, p, 1) == -10
+    fpar = (ctypes.c_float * 5)(-1.0, 1.0, 0.0, 0.0, 1.0)
+    bad_flag = (ctypes.c_float * 5)(3.0, 1.0, 0.0, 0.0, 1.0)
+    assert h.b2_srotm(c, -1, p, 1, p, 1, ctypes.cast(fpar, ctypes.c_void_p)) == -1
+    assert h.b2_srotm(c, 4, p, 1, p, 0, ctypes.cast(fpar, ctypes.c_void_p)) == -5
+    assert h.b2_srotm(c, 4, p, 1, p, 1, None) == -6
+    assert h.b2_srotm(c, 4, p, 1, p, 1, ctypes.cast(bad_flag, ctypes.c_void_p)) == -6
+    assert h.b2_dsdot(c, 4, p, 1, p, 1, None) == -6
+    assert h.b2_sdsdot(c, 4, 0.0, p, 1, p, 0, p) == -6
+    assert h.b2_sdsdot(c, 4, 0.0, p, 1, p, 1, None) == -7
     # context checks come after argument checks and before any launch
     assert h.b2_saxpy(None, 4, 1.0, p, 1, p, 1) == b2.STATUS_BAD_CONTEXT
     bad = b2.B2Ctx(None, 0x1001, 1 << 20, None, 0)
