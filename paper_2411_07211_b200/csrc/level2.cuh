@@ -17,6 +17,8 @@
 // order and applies alpha / beta.  No atomics: results are bit-reproducible.
 #pragma once
 
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace b2 {
@@ -485,7 +487,17 @@ static L2Plan plan_rowout(const L2Args<T>& a, bool narrow_ok) {
   p.shape = nv >= 128 ? SHAPE_WIDE : (nv > 16 || !narrow_ok) ? SHAPE_MID : nv > 8 ? SHAPE_HALF : SHAPE_QUARTER;
   const int64_t tile_bytes = (int64_t)shape_rb(p.shape) * shape_packs_per_row(p.shape) * V * sizeof(T);
   int64_t cpc = knob(kKnobGemvNTileBytes) / tile_bytes;
-  p.ctiles_per_cta = (int)(cpc < 1 ? 1 : cpc);
+  if (cpc < 1) cpc = 1;
+  // A matrix of a few long rows (at most 8 row steps) would get one partial per column split
+  // and a finalize pass that adds thousands of them per row: there the splits are limited to
+  // about eight resident blocks per SM in all.
+  const int64_t nrs = (a.rows + shape_rb(p.shape) - 1) / shape_rb(p.shape);
+  if (nrs <= 8) {
+    const int64_t nct = (nv + shape_packs_per_row(p.shape) - 1) / shape_packs_per_row(p.shape);
+    const int64_t want_ncs = std::max<int64_t>(1, (int64_t)sm_count() * 8 / nrs);
+    cpc = std::max(cpc, (nct + want_ncs - 1) / want_ncs);
+  }
+  p.ctiles_per_cta = (int)cpc;
   p.rows_per_cta = shape_rb(p.shape);
   return p;
 }
@@ -496,6 +508,8 @@ static L2Plan plan_colout(const L2Args<T>& a, bool narrow_ok, int64_t rows_per_c
   const int64_t nv = (a.cols + V - 1) / V;
   L2Plan p;
   p.shape = (nv > 16 || !narrow_ok) ? SHAPE_MID : nv > 8 ? SHAPE_HALF : SHAPE_QUARTER;
+  // element-wise rows (not 16-byte aligned): a 32-element column tile makes tiny blocks, take 128
+  if (V == 1 && nv >= 128) p.shape = SHAPE_WIDE;
   p.ctiles_per_cta = 1;
   if ((a.rows + rows_per_cta - 1) / rows_per_cta > 1024) rows_per_cta = (a.rows + 1023) / 1024;
   p.rows_per_cta = rows_per_cta;
