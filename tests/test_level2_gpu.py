@@ -51,7 +51,8 @@ GEMV_SHAPES = [(1, 1), (3, 5), (17, 33), (64, 64), (100, 700), (700, 100), (257,
 def test_gemv(b2, ctx, dtype, order, trans, m, n):
     minor, major = (n, m) if order == orc.ROW_MAJOR else (m, n)
     lenx, leny = (n, m) if trans == orc.NO_TRANS else (m, n)
-    cases = [(0, 0, 1, 1, 0.5), (0, 0, 1, 1, 0.0), (1, 0, 2, 2, 0.5), (4, 1, -1, 3, 0.0), (3, 0, 1, -2, 0.5)]
+    cases = [(0, 0, 1, 1, 0.5), (0, 0, 1, 1, 0.0), (1, 0, 2, 2, 0.5), (4, 1, -1, 3, 0.0), (3, 0, 1, -2, 0.5),
+             (0, 0, -2, 3, 0.5)]  # unpadded with strided vectors: the narrow-matrix kernels see every increment
     for pad, offset, incx, incy, beta in cases:
         lda = minor + pad
         a = matbuf(m * 31 + n, major, minor, lda, dtype)
@@ -84,7 +85,7 @@ def test_gemv(b2, ctx, dtype, order, trans, m, n):
 @pytest.mark.parametrize("m,n", GEMV_SHAPES)
 def test_ger(b2, ctx, dtype, order, m, n):
     minor, major = (n, m) if order == orc.ROW_MAJOR else (m, n)
-    for pad, offset, incx, incy in [(0, 0, 1, 1), (1, 0, 2, 2), (4, 1, -1, 3), (2, 0, 1, -2)]:
+    for pad, offset, incx, incy in [(0, 0, 1, 1), (1, 0, 2, 2), (4, 1, -1, 3), (2, 0, 1, -2), (0, 0, -1, 2)]:
         lda = minor + pad
         a = matbuf(m * 17 + n, major, minor, lda, dtype)
         x = synth.vector_np(3, m + n, m, dtype)
