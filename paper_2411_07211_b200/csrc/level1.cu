@@ -149,8 +149,12 @@ __global__ void __launch_bounds__(kThreads) l1_map_strided(Op op, T* __restrict_
       a[k] = T(0);
       b[k] = T(0);
       if (i < n) {
-        if (Op::RX) a[k] = __ldcs(x + i * incx);
-        if (Op::RY) b[k] = __ldcs(y + i * incy);
+        // An array that is written back must not be loaded evict-first: a strided store covers
+        // only part of a sector, and the rest has to be still in L2 when it arrives, or the sector
+        // is fetched from DRAM a second time (measured with L2 full of clean lines: swap with
+        // increment 2 at 0.77 of the copy rate evict-first, 1.00 without).
+        if (Op::RX) a[k] = Op::WX ? __ldcg(x + i * incx) : __ldcs(x + i * incx);
+        if (Op::RY) b[k] = Op::WY ? __ldcg(y + i * incy) : __ldcs(y + i * incy);
       }
     }
 #pragma unroll
