@@ -153,6 +153,8 @@ __global__ void __launch_bounds__(kThreads) l1_map_strided(Op op, T* __restrict_
         // only part of a sector, and the rest has to be still in L2 when it arrives, or the sector
         // is fetched from DRAM a second time (measured with L2 full of clean lines: swap with
         // increment 2 at 0.77 of the copy rate evict-first, 1.00 without).
+        // a write-only strided target: start the fill of its sectors now, not when the store arrives
+        if (!Op::RY && Op::WY) asm volatile("prefetch.global.L2 [%0];" ::"l"(y + i * incy));
         if (Op::RX) a[k] = Op::WX ? __ldcg(x + i * incx) : __ldcs(x + i * incx);
         if (Op::RY) b[k] = Op::WY ? __ldcg(y + i * incy) : __ldcs(y + i * incy);
       }
