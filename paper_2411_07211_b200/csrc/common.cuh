@@ -54,6 +54,21 @@ __device__ __forceinline__ Pack<T, N> ld_cs(const T* p) {
   return r;
 }
 
+// Streaming load of data that this kernel writes back: L2 only, normal eviction priority, so
+// that the line is still there when the store arrives (see ld_cs for the evict-first form).
+template <typename T, int N>
+__device__ __forceinline__ Pack<T, N> ld_cg(const T* p) {
+  Pack<T, N> r;
+  if constexpr (sizeof(T) * N == 16) {
+    uint4 t = __ldcg(reinterpret_cast<const uint4*>(p));
+    r = *reinterpret_cast<Pack<T, N>*>(&t);
+  } else {
+    static_assert(N == 1, "packs are 16 bytes or one element");
+    r.v[0] = __ldcg(p);
+  }
+  return r;
+}
+
 // Read-only streaming load (data not written by this kernel): non-coherent path, no L1
 // allocation so the matrix stream does not evict the reused vectors.
 template <typename T, int N>
