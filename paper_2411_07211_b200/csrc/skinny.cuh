@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(kThreads, 3) skinny_ger_kernel(T* __restrict__
 #pragma unroll
       for (int g = 0; g < kSkinnyGroup; ++g) {
         const int pos = (k0 + g) * 32 + lane;
-        if (k0 + g < ppr && pos < npacks) av[g] = ld_cs<T, V>(reinterpret_cast<const T*>(dst + pos));
+        if (k0 + g < ppr && pos < npacks) av[g] = ld_cg<T, V>(reinterpret_cast<const T*>(dst + pos));
       }
 #pragma unroll
       for (int g = 0; g < kSkinnyGroup; ++g) {
