@@ -5,8 +5,8 @@ A "step" is one pass over the whole variant cross-product (every routine x {f32,
 trans/uplo/diag options x inc in {1, 2}), each variant sized to a 256 MiB working set.  Every
 variant is timed with its own pair of CUDA events on the launching stream; every working set
 is larger than L2 and L2 is additionally swept (256 MiB read-only pass) before each variant,
-so no number is an L2-resident one.  Prints ONE JSON
-line (rank 0).
+so no number is an L2-resident one.  Rank 0 prints ONE short JSON line (summary keys only) as
+the last line of stdout; the per-variant rows go to a table file (--table).
 
     python bench.py --gpus 1 --steps 20 --warmup 3
     python bench.py --impl reference        # the CPU oracle on the host cores (bounded sample)
@@ -28,12 +28,17 @@ sys.path.insert(0, ROOT)
 MIB = 1 << 20
 ROW, COL, NOTR, TR, UP, LO, NONU, UNIT = 101, 102, 111, 112, 121, 122, 131, 132
 FALLBACK_PEAK_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of each kernel template at the bench
-# sizes, from the ncu captures summarised in profiles/kernels_config5_ncu_full.md (same kernels).
-# Set an entry to None when its kernel changes and the counters have not been retaken.
-# trsv: the sub-block kernel, which serves every bench variant (273.4-274.0 MB float, 275.3 MB double).
-NCU_DRAM_BYTES_PER_LAUNCH = {"trsv": 274.0e6, "l2_tile": 271.3e6, "l1_reduce": 272.3e6, "l1_map": 351.8e6,
-                             "ger": 479.3e6}
+
+
+def ncu_dram_bytes_per_launch():
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of each kernel template at the
+    bench sizes, as recorded beside the ncu summaries (one entry per kernel family; null once a
+    kernel has changed and its counters have not been retaken)."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "ncu_dram_bytes_per_launch.json")) as f:
+            return json.load(f)["bytes_per_launch"]
+    except Exception:
+        return {}
 
 
 # --------------------------------------------------------------------------- variant table
@@ -494,6 +499,27 @@ def aggregate(specs, med_ms, world, peak):
 
 
 # --------------------------------------------------------------------------- main
+def _short(v, digits=4):
+    """Floats to `digits` significant digits, recursively (keeps the printed line short)."""
+    if isinstance(v, float):
+        return float(f"{v:.{digits}g}")
+    if isinstance(v, dict):
+        return {k: _short(x, digits) for k, x in v.items()}
+    if isinstance(v, (list, tuple)):
+        return [_short(x, digits) for x in v]
+    return v
+
+
+def final_line(out: dict) -> str:
+    """The ONE line printed last: the summary keys only, floats shortened.  Per-variant rows never
+    go here (they are written to the table file): a reader that keeps only the end of stdout must
+    still see the whole line."""
+    keep = {k: v for k, v in out.items() if k not in ("variants", "next_rows")}
+    line = json.dumps(_short(keep, 5), separators=(",", ":"))
+    assert len(line) < 4096, f"final line too long ({len(line)} bytes)"
+    return line
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -506,7 +532,8 @@ def main():
                                                    "strings (tuning runs; the headline run uses all)")
     ap.add_argument("--next-only", action="store_true", help="time only the rows built after the headline set "
                                                              "(--filter then selects among those)")
-    ap.add_argument("--table", default=None, help="also write the per-variant table (JSON) to this path")
+    ap.add_argument("--table", default=None, help="where the per-variant table (JSON) is written "
+                                                  "(default: bench_table.json in the run's output folder)")
     args = ap.parse_args()
     if args.impl == "reference":
         reference_arm(args)
@@ -580,7 +607,7 @@ def main():
                      "share_of_time": v["ms"] / sum(x["ms"] for x in fam.values()), "variants": v["launches"]}
                  for k, v in fam.items()}
     dom = max(fam, key=lambda k: fam[k]["ms"])
-    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(dom)
+    traffic = ncu_dram_bytes_per_launch().get(dom)
     roofline = {"bound": "hbm", "kernel": dom, "achieved": by_kernel[dom]["achieved"], "peak": peak, "unit": "GB/s",
                 "frac": by_kernel[dom]["frac"], "traffic": traffic, "peak_source": peak_src,
                 "by_kernel": by_kernel}
@@ -614,14 +641,16 @@ def main():
                                          f"({time.perf_counter() - t0:.1f} s of CPU work)"}
     else:
         out["cpu_baseline"] = None
-    out["variants"] = [{k: (round(v, 4) if isinstance(v, float) else v) for k, v in r.items()} for r in rows]
+    table = dict(out)
+    table["variants"] = [{k: (round(v, 4) if isinstance(v, float) else v) for k, v in r.items()} for r in rows]
     if world == 1 and not args.filter:
-        out["next_rows"] = next_rows_leg(wl, min(args.steps, 10), peak)
-    if args.table:
-        os.makedirs(os.path.dirname(os.path.abspath(args.table)), exist_ok=True)
-        with open(args.table, "w") as f:
-            json.dump(out, f, indent=1)
-    print(json.dumps(out))
+        table["next_rows"] = next_rows_leg(wl, min(args.steps, 10), peak)
+        out["next_rows_geomean_frac"] = table["next_rows"]["geomean_frac"]
+    path = args.table or os.path.join(ROOT, "gpurun_out", "bench_table.json")
+    os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+    with open(path, "w") as f:
+        json.dump(table, f, indent=1)
+    print(final_line(out))
     if world > 1:
         dist.destroy_process_group()
 

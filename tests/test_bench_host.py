@@ -59,3 +59,41 @@ def test_max_over_ranks_two_gloo_processes():
         p.join(timeout=60)
         assert p.exitcode == 0
     assert res[0] == res[1] == [2.0, 5.0, 2.0]
+
+
+def test_final_line_is_short_and_keeps_the_summary_keys():
+    """The last stdout line must survive a reader that keeps only the end of the output: summary
+    keys only, no per-variant rows, well under 4 KB even with all 120 variants aggregated."""
+    import json
+    specs = bench.variant_specs()
+    rows, value = bench.aggregate(specs, [0.05 + 0.001 * k for k in range(len(specs))], world=1, peak=6547.2)
+    fams = sorted({sp["family"] for sp in specs})
+    by_kernel = {k: {"achieved": 5269.388006569296, "frac": 0.8048307683543034, "share_of_time": 0.2382904333518465,
+                     "variants": 48} for k in fams}
+    out = {
+        "metric": "achieved HBM GB/s per BLAS-1/2 variant, geomean over variants", "value": value, "unit": "GB/s",
+        "n_gpus": 1, "steps": 20, "warmup": 3, "ms_per_step": 16.193397521972656, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32+f64", "data": "synthetic",
+        "config": {"workload": "w" * 120, "variants": 120, "l2": "x" * 220, "bytes": "touched sectors (span bytes)",
+                   "parallelism": "single GPU"},
+        "geomean_frac_of_peak": 0.6152370341687622, "geomean_frac_of_peak_without_trsv": 0.8522784166663647,
+        "geomean_frac_by_family": {k: 0.9382842251889021 for k in fams}, "min_variant": "trsv_unn_f64_inc1",
+        "gpu_launches": 7040, "clocks": {"sm_mhz": 1965.0, "sm_max_mhz": 1965.0, "reasons": [], "samples": 2},
+        "roofline": {"bound": "hbm", "kernel": "trsv", "achieved": 1640.9586225995336, "peak": 6547.2, "unit": "GB/s",
+                     "frac": 0.2506351757391761, "traffic": 274000000.0,
+                     "peak_source": "measured (MEASURED_PEAKS.json hbm_gbs)", "by_kernel": by_kernel},
+        "e2e": {"value": 36.17699841312217, "unit": "GB/s (geomean over variants, host buffers in and out)",
+                "h2d_bytes_per_step": 50775709228, "d2h_bytes_per_step": 5369180156, "steps": 2},
+        "cpu_baseline": {"value": 1.313513313524947, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": "s" * 100},
+        "variants": rows, "next_rows": {"variants": rows},
+    }
+    line = bench.final_line(out)
+    assert "\n" not in line and len(line) < 4096
+    back = json.loads(line)
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "roofline", "cpu_baseline",
+                "e2e", "clocks", "gpu_launches", "config"):
+        assert key in back, key
+    assert "variants" not in back and "next_rows" not in back
+    assert back["value"] == pytest.approx(value, rel=1e-4)
+    assert back["e2e"]["h2d_bytes_per_step"] == 50775709228  # integers are kept whole
+    assert set(back["roofline"]["by_kernel"]) == set(fams)
