@@ -264,7 +264,10 @@ def test_gemv_ger_bruteforce(dtype, order, m, n, pad):
             absterms = orc.gemv(order, trans, m, n, alpha, a, lda, strided(x, incx), incx, b, by, incy)
             exact = [fa * v + (fbeta * w if b != 0 else 0) for v, w in zip(matvec(op, fr(x)), fr(y))]
             assert_within_ulp(logical(by, leny, incy), exact, dtype)
-            assert np.all(absterms >= np.abs(logical(by, leny, incy)).astype(np.float64) * (1 - 1e-6))
+            # the tolerance scale itself: sum of |alpha*a*x| over the row plus |beta*y|, exactly
+            want_abs = [float(sum((abs(fa * a_ * x_) for a_, x_ in zip(row, fr(x))), Fraction(0))
+                              + (abs(fbeta * w) if b != 0 else 0)) for row, w in zip(op, fr(y))]
+            assert np.allclose(absterms, want_abs, rtol=1e-12, atol=0)
         # alpha == 0 => y = beta*y exactly, A and x never matter
         by = strided(y, incy)
         orc.gemv(order, trans, m, n, dtype(0), np.full_like(a, np.nan), lda,
@@ -324,7 +327,9 @@ def test_symv_bruteforce(dtype, order, uplo, n, pad):
         exact = [Fraction(float(alpha)) * v + Fraction(float(beta)) * w
                  for v, w in zip(matvec(sym, fr(x)), fr(y))]
         assert_within_ulp(logical(by, n, incy), exact, dtype)
-        assert np.all(np.isfinite(absterms))
+        want_abs = [float(sum((abs(Fraction(float(alpha)) * a_ * x_) for a_, x_ in zip(row, fr(x))), Fraction(0))
+                          + abs(Fraction(float(beta)) * w)) for row, w in zip(sym, fr(y))]
+        assert np.allclose(absterms, want_abs, rtol=1e-12, atol=0)
         # symv == gemv on the explicitly symmetrised dense matrix (same oracle arithmetic)
         full = np.array([[float(v) for v in row] for row in sym], dtype=dtype).ravel()
         by2 = strided(y, incy)
@@ -348,20 +353,30 @@ def test_trmv_trsv_bruteforce(dtype, order, uplo, trans, diag, n, pad):
         bx = strided(x, incx)
         absterms = orc.trmv(order, uplo, trans, diag, n, a, lda, bx, incx)
         assert_within_ulp(logical(bx, n, incx), matvec(op, fr(x)), dtype)
-        assert np.all(np.isfinite(absterms))
+        want_abs = [float(sum((abs(e * v) for e, v in zip(row, fr(x))), Fraction(0))) for row in op]
+        assert np.allclose(absterms, want_abs, rtol=1e-12, atol=0)
         # trsv against exact Gauss-Jordan elimination of the dense op(A)
         bx = strided(x, incx)
-        orc.trsv(order, uplo, trans, diag, n, a, lda, bx, incx)
+        absterms = orc.trsv(order, uplo, trans, diag, n, a, lda, bx, incx)
         exact = gauss_solve(op, fr(x))
         got = logical(bx, n, incx)
         for g, e in zip(got, exact):
             assert abs(float(g) - float(e)) <= 4 * eps * max(abs(float(e)), 1e-30) + 0, (g, float(e))
+        # row balance |b_i| + sum over the OFF-diagonal entries of |op(A)_ij x_j|, with the exact
+        # solution (the oracle's own wide solution differs from it far below 1e-12 here)
+        want_abs = [float(abs(b) + sum((abs(op[i][j] * exact[j]) for j in range(n) if j != i), Fraction(0)))
+                    for i, b in enumerate(fr(x))]
+        assert np.allclose(absterms, want_abs, rtol=1e-12, atol=0)
         # residual helper agrees with an exact evaluation
         resid, scale = orc.trsv_residual(order, uplo, trans, diag, n, a, lda, strided(x, incx), incx,
                                          bx, incx)
         ex_res = [abs(b - v) for b, v in zip(fr(x), matvec(op, fr(got)))]
         weps = 2.0 ** -52 if dtype == np.float32 else 2.0 ** -63  # rounding unit of W
         assert np.all(np.abs(resid - np.array([float(v) for v in ex_res])) <= 8 * weps * scale)
+        # scale_i = |b_i| + sum_j |op(A)_ij xs_j| over the whole row (diagonal included), exactly
+        want_scale = [float(abs(b) + sum((abs(e * v) for e, v in zip(row, fr(got))), Fraction(0)))
+                      for b, row in zip(fr(x), op)]
+        assert np.allclose(scale, want_scale, rtol=1e-12, atol=0)
         assert np.all(resid <= 2 * eps * scale)
         # trsv(trmv(x)) recovers x
         bx = strided(x, incx)

@@ -4,14 +4,16 @@ Some users of the library run where no device memory can be had at call time: in
 application whose own allocator has taken the whole GPU heap, or in a loop that must never
 block on cudaMalloc.  For them the library keeps the reduction's scratch in a fixed array of
 its own.  This test calls that entry point through the C ABI twice in a row (the second call
-finds the first call's leftovers in the shared array) and compares each result with the
-ordinary b2_sdot on the same inputs, under the tolerance of the other reduction tests.
+finds the first call's leftovers in the shared array) and compares each result with the CPU
+oracle's dot product and with the ordinary b2_sdot on the same inputs, under the tolerance of
+the other reduction tests (2e-6 x the oracle's sum of |x_i y_i|).
 Collected last on purpose: a run that stops at the first failure has then run everything else.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import blas_oracle as orc
 from paper_2411_07211_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -31,12 +33,10 @@ def test_sdot_noalloc_matches_sdot_twice_in_a_row():
         got = torch.full((2,), float("nan"), dtype=torch.float32, device="cuda")
         b2.dot(ctx, n, x, incx, y, incy, want)
         b2.sdot_noalloc(n, x, incx, y, incy, got[0:1])
-        xs = x[::abs(incx)][:n].double()
-        ys = y[::abs(incy)][:n].double()
-        if (incx < 0) != (incy < 0):
-            ys = ys.flip(0)
-        absterms = float((xs * ys).abs().sum().item())
+        ref, absterms = orc.dot(n, np.ascontiguousarray(x.cpu().numpy()), incx,
+                                np.ascontiguousarray(y.cpu().numpy()), incy)
         g = got.cpu().numpy()
+        assert abs(float(g[0]) - float(ref)) <= 2e-6 * absterms, (call, g[0], ref)
         assert abs(float(g[0]) - float(want.item())) <= 2e-6 * absterms, (call, g[0], want.item())
         assert np.isnan(g[1])  # the word after the result is not touched
 
