@@ -95,16 +95,20 @@ def peak_gbs():
 
 # --------------------------------------------------------------------------- clocks sampler
 class ClockSampler:
+    """nvidia-smi polled every 50 ms from before the warm-up; `stop` summarises the samples that
+    fall inside the timed region (marked by `mark_start` / `mark_end`), and when the region is too
+    short to hold three of them, the samples taken from the warm-up on (the same load)."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.proc = None
-        self.lines = []
+        self.lines = []  # (arrival time, text)
+        self.t_load = self.t0 = self.t1 = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except Exception:
@@ -112,33 +116,56 @@ class ClockSampler:
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.monotonic(), line.strip()))
+
+    def wait_first(self, timeout=10.0):
+        """Blocks until the first sample has arrived (nvidia-smi takes a moment to start)."""
+        t_end = time.monotonic() + timeout
+        while self.proc is not None and not self.lines and time.monotonic() < t_end:
+            time.sleep(0.02)
+
+    def mark_load(self):
+        self.t_load = time.monotonic()
+
+    def mark_start(self):
+        self.t0 = time.monotonic()
+
+    def mark_end(self):
+        self.t1 = time.monotonic()
+
+    @staticmethod
+    def summarise(lines, t_load, t0, t1):
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        parsed = []
+        for t, line in lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                parsed.append((t, float(parts[0]), float(parts[1]),
+                               [nm for nm, val in zip(names, parts[2:6]) if val.lower().startswith("active")]))
+            except ValueError:
+                continue
+        inside = [r for r in parsed if t0 is not None and t1 is not None and t0 <= r[0] <= t1 + 0.05]
+        window = "timed region"
+        if len(inside) < 3:
+            inside = [r for r in parsed if t_load is None or t1 is None or t_load <= r[0] <= t1 + 0.05]
+            window = "warm-up and timed region (the timed region alone is shorter than three samples)"
+        sm = sorted(r[1] for r in inside)
+        reasons = sorted({nm for r in inside for nm in r[3]})
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": inside[-1][2] if inside else None,
+                "reasons": reasons, "samples": len(sm), "window": window}
 
     def stop(self):
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
+        time.sleep(0.06)  # one more sample that still belongs to the region
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], None, set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 6:
-                continue
-            try:
-                sm.append(float(parts[0]))
-                mx = float(parts[1])
-            except ValueError:
-                continue
-            for nm, val in zip(names, parts[2:6]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(sm)}
+        return self.summarise(list(self.lines), self.t_load, self.t0, self.t1)
 
 
 # --------------------------------------------------------------------------- GPU arm
@@ -561,6 +588,10 @@ def main():
     wl = GpuWorkload(device, args.filter)
     nv = len(wl.specs)
     warm = max(3, args.warmup)
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.wait_first()
+        sampler.mark_load()
     for _ in range(warm):
         wl.step()
     torch.cuda.synchronize(device)
@@ -569,7 +600,8 @@ def main():
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize(device)
-    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.mark_start()
     launches0 = b2.launch_count()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record()
@@ -577,6 +609,8 @@ def main():
         wl.step(events[s])
     t_end.record()
     torch.cuda.synchronize(device)
+    if sampler:
+        sampler.mark_end()
     if world > 1:
         dist.barrier()
     launches = b2.launch_count() - launches0

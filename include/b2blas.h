@@ -62,7 +62,10 @@ enum {
  *                   level-2 calls; b2_workspace_bytes() is a comfortable default.
  *   device_status   optional device int.  trsv writes B2_STATUS_TIMEOUT there if a bounded
  *                   wait on another thread block ran out (the call's output is then invalid).
- *                   Never written otherwise; the caller zeroes it.
+ *                   Never written otherwise; the caller zeroes it.  A timed-out call leaves
+ *                   the control block dirty: call b2_workspace_reset before the workspace is
+ *                   used again.  A trsv call that finds the control block dirty solves
+ *                   nothing and writes B2_STATUS_TIMEOUT again.
  *   wait_limit      polling iterations before a trsv wait gives up; 0 = library default.
  */
 typedef struct b2_ctx {
@@ -74,7 +77,15 @@ typedef struct b2_ctx {
 } b2_ctx;
 
 size_t b2_workspace_min_bytes(void); /* control block + level-1 partials                   */
-size_t b2_workspace_bytes(void);     /* recommended size (64 MiB)                           */
+/* Recommended size (64 MiB): a default, not a bound.  It serves every call on matrices up to
+ * 32768 x 32768 and vectors of any length without B2_STATUS_WORKSPACE_TOO_SMALL; the exact
+ * need of one call is b2_workspace_query's. */
+size_t b2_workspace_bytes(void);
+/* Smallest workspace size with which no routine of this library returns
+ * B2_STATUS_WORKSPACE_TOO_SMALL on an m x n matrix (vectors of max(m, n) elements; level-1
+ * calls: pass m = n = 1) of elem_bytes-sized elements (4 or 8).  Larger workspaces only allow
+ * finer work splitting.  Returns 0 for a negative size or another element size. */
+size_t b2_workspace_query(int64_t m, int64_t n, size_t elem_bytes);
 int b2_workspace_reset(const b2_ctx* ctx); /* async memset of the control block to zero     */
 const char* b2_status_string(int status);
 int b2_version(void);

@@ -93,6 +93,8 @@ def lib():
             fn.restype = _int
         h.b2_workspace_min_bytes.restype = ctypes.c_size_t
         h.b2_workspace_bytes.restype = ctypes.c_size_t
+        h.b2_workspace_query.restype = ctypes.c_size_t
+        h.b2_workspace_query.argtypes = [_i64, _i64, ctypes.c_size_t]
         h.b2_status_string.restype = ctypes.c_char_p
         h.b2_status_string.argtypes = [_int]
         h.b2_version.restype = _int
@@ -106,7 +108,7 @@ def lib():
 
 
 def exported_symbols():
-    return sorted(_protos().keys()) + ["b2_workspace_min_bytes", "b2_workspace_bytes", "b2_status_string",
+    return sorted(_protos().keys()) + ["b2_workspace_min_bytes", "b2_workspace_bytes", "b2_workspace_query", "b2_status_string",
                                        "b2_version", "b2_launch_count", "b2_set_tuning", "b2_get_tuning"]
 
 

@@ -40,6 +40,16 @@ extern "C" {
 size_t b2_workspace_min_bytes(void) { return b2::kCtlBytes + 64 * 1024; }
 size_t b2_workspace_bytes(void) { return (size_t)64 << 20; }
 
+size_t b2_workspace_query(int64_t m, int64_t n, size_t elem_bytes) {
+  if (m < 0 || n < 0 || (elem_bytes != 4 && elem_bytes != 8)) return 0;
+  // level 1: one partial per block of the reduction grid; level 2 with every split merged: one
+  // row of partials per output vector; trsv: one or two tagged 64-bit words per unknown
+  const size_t vec = (size_t)(m > n ? m : n);
+  const size_t level2 = ((size_t)m + (size_t)n) * elem_bytes + 1024;
+  const size_t trsv = vec * 8 * (elem_bytes / 4);
+  return b2_workspace_min_bytes() + (level2 > trsv ? level2 : trsv);
+}
+
 int b2_workspace_reset(const b2_ctx* ctx) {
   b2::Launch l;
   if (int st = b2::make_launch(ctx, &l)) return st;

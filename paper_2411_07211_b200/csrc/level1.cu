@@ -507,15 +507,27 @@ __global__ void sdsdot_finish(const double* __restrict__ acc, float sb, float* _
 static int grid_cap() { return sm_count() * (int)knob(kKnobL1BlocksPerSm); }
 
 // One resident wave: as many blocks as really fit (the kernel grid-strides over the data), so
-// no second, partly filled wave trails behind.
+// no second, partly filled wave trails behind.  Only the blocks-per-SM figure of the kernel is
+// cached (per device id); the SM count, the knob and the cap are read on every call.
+struct WaveCache {
+  int per_sm[64] = {0};
+};
 template <class Kernel>
-static int one_wave(Kernel kernel, int cap) {
-  int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm <= 0) {
+static int one_wave(Kernel kernel, int cap, WaveCache& cache) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
     (void)cudaGetLastError();
     return cap;
   }
-  const int wave = per_sm * sm_count();
+  if (cache.per_sm[dev] == 0) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm <= 0) {
+      (void)cudaGetLastError();
+      return cap;
+    }
+    cache.per_sm[dev] = per_sm;
+  }
+  const int wave = cache.per_sm[dev] * sm_count();
   return wave < cap ? wave : cap;
 }
 
@@ -575,7 +587,8 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
     if (head > n) head = n;
     const int64_t nvec = (n - head) / V;
     const int64_t nchunks = (nvec + kThreads * NV - 1) / (kThreads * NV);
-    static const int wave = one_wave(l1_reduce_unit<T, Op, NV>, cap);
+    static WaveCache wc;
+    const int wave = one_wave(l1_reduce_unit<T, Op, NV>, cap, wc);
     const int64_t grid = nchunks < 1 ? 1 : (nchunks > wave ? wave : nchunks);
     l1_reduce_unit<T, Op, NV><<<(unsigned)grid, kThreads, 0, l.stream>>>(x, Op::RY ? y : x, n, head, nvec, nchunks,
                                                                         partials, ticket, result);
@@ -586,14 +599,16 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
     if (head > span) head = span;
     const int64_t nvec = (span - head) / V;
     const int64_t nchunks = (nvec + kThreads * NV - 1) / (kThreads * NV);
-    static const int wave = one_wave(l1_reduce_unit<T, Op, NV, 2>, cap);
+    static WaveCache wc;
+    const int wave = one_wave(l1_reduce_unit<T, Op, NV, 2>, cap, wc);
     const int64_t grid = nchunks < 1 ? 1 : (nchunks > wave ? wave : nchunks);
     l1_reduce_unit<T, Op, NV, 2><<<(unsigned)grid, kThreads, 0, l.stream>>>(x, Op::RY ? y : x, span, head, nvec, nchunks,
                                                                            partials, ticket, result);
   } else {
     constexpr int NE = Op::RY ? 8 : 16;
     const int64_t nchunks = (n + kThreads * NE - 1) / (kThreads * NE);
-    static const int wave = one_wave(l1_reduce_strided<T, Op, NE>, cap);
+    static WaveCache wc;
+    const int wave = one_wave(l1_reduce_strided<T, Op, NE>, cap, wc);
     const int64_t grid = nchunks > wave ? wave : nchunks;
     l1_reduce_strided<T, Op, NE><<<(unsigned)grid, kThreads, 0, l.stream>>>(
         vec_base(x, n, incx), incx, Op::RY ? vec_base(y, n, incy) : x, Op::RY ? incy : 1, n, nchunks, partials, ticket,

@@ -51,11 +51,15 @@ __device__ __forceinline__ unsigned long long ld_word(const unsigned long long* 
 __device__ __forceinline__ void st_word(unsigned long long* p, unsigned long long v) {
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
+// Named barriers.  The polling loop in front of them lets lanes leave at different iterations, so
+// the warp is re-converged first and the forms that count threads (not whole warps) are used.
 __device__ __forceinline__ void bar_sync(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+  __syncwarp();
+  asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 __device__ __forceinline__ void bar_arrive(int id, int count) {
-  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+  __syncwarp();
+  asm volatile("barrier.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
 template <typename T>
@@ -131,7 +135,7 @@ __device__ __forceinline__ double decode(const unsigned long long* w, double) {
 
 // COLTYPE: op(A)'s rows are columns of the stored row-major view.  BACKWARD: solve bottom-up.
 // NB = unknowns per thread block: 128 for float, 64 for double (the diagonal-block work grows with
-// NB^2 per unknown and double-precision multiply-adds are scarce on this part).
+// NB^2 per unknown, and a 128 x 128 double block with its inverse would not fit in shared memory).
 template <typename T, int NB, int V, bool COLTYPE, bool BACKWARD, bool UNIT>
 __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
   // A tile is NB own unknowns x 64 source unknowns; in memory it is NB rows x 64 columns

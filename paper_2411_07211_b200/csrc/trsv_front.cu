@@ -286,6 +286,9 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     if (rank == 0u && ct == 0) {
       unsigned kk = 0xffffffffu;
       if (!wt.dead && ld_flag(wt.abort_word) == 0u) kk = atomicAdd(p.ctl + kCtlTrsvTicket, 1u);
+      // abort word up (raised in this call, or left by an earlier timed-out call on a workspace
+      // that was not reset): nothing more is solved, and the caller must be able to see that
+      else if (p.device_status) atomicExch(p.device_status, (int)B2_STATUS_TIMEOUT);
       if (CS > 1) {
         for (unsigned r = 0; r < (unsigned)CS; ++r) st_remote_u32(map_remote(&s_ticket[parity], r), kk);
       } else {

@@ -27,6 +27,10 @@ def test_header_symbols_exported(b2):
     assert set(b2.exported_symbols()) == set(declared)
     assert b2.lib().b2_version() >= 100
     assert b2.lib().b2_workspace_bytes() >= b2.lib().b2_workspace_min_bytes() > 4096
+    q = b2.lib().b2_workspace_query
+    assert q(1, 1, 4) >= b2.lib().b2_workspace_min_bytes() and q(-1, 1, 4) == 0 and q(1, 1, 3) == 0
+    assert q(32768, 32768, 8) <= b2.lib().b2_workspace_bytes()  # the default serves the largest config
+    assert q(1 << 20, 64, 8) >= ((1 << 20) + 64) * 8 and q(70000, 70000, 8) >= 70000 * 16
     assert b"ok" == b2.lib().b2_status_string(0)
     assert b"argument" in b2.lib().b2_status_string(-3)
 

@@ -97,3 +97,17 @@ def test_final_line_is_short_and_keeps_the_summary_keys():
     assert back["value"] == pytest.approx(value, rel=1e-4)
     assert back["e2e"]["h2d_bytes_per_step"] == 50775709228  # integers are kept whole
     assert set(back["roofline"]["by_kernel"]) == set(fams)
+
+
+def test_clock_summary_windows():
+    """Samples inside the timed region are used when there are at least three; a shorter region
+    falls back to everything from the warm-up on, and slowdown reasons are collected."""
+    mk = lambda t, mhz, flags="Not Active, Not Active, Not Active, Not Active": (t, f"{mhz}, 1965, {flags}")
+    lines = [mk(0.0, 300), mk(1.0, 1900), mk(1.1, 1950), mk(2.0, 1965), mk(2.05, 1965), mk(2.1, 1960),
+             mk(2.15, 1965, "Not Active, Not Active, Not Active, Active")]
+    out = bench.ClockSampler.summarise(lines, t_load=0.9, t0=1.95, t1=2.2)
+    assert out["samples"] == 4 and out["sm_mhz"] == 1965 and out["sm_max_mhz"] == 1965
+    assert out["reasons"] == ["sw_power_cap"] and out["window"] == "timed region"
+    out = bench.ClockSampler.summarise(lines, t_load=0.9, t0=2.12, t1=2.2)  # one sample inside: widen
+    assert out["samples"] == 6 and out["window"].startswith("warm-up") and out["sm_mhz"] == 1965
+    assert bench.ClockSampler.summarise([], None, None, None)["sm_mhz"] is None

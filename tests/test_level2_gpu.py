@@ -198,7 +198,15 @@ def test_trsv_bounded_wait_reports_timeout(b2):
         assert ctx.device_status() == b2.STATUS_TIMEOUT
     finally:
         b2.set_tuning(b2.KNOB_TRSV_DEBUG_SKIP, -1)
-    ctx.reset()  # a timed-out call leaves the control block dirty
+    # a timed-out call leaves the control block dirty: without a reset the next call must say so
+    # (and leave x as it was) instead of returning an unsolved vector with status 0
+    ctx.status.zero_()
+    x = Guarded(synth.vector_np(1, 1, n, np.float32))
+    b2.trsv(ctx, orc.ROW_MAJOR, orc.LOWER, orc.NO_TRANS, orc.NON_UNIT, n, a.t, n, x.t, 1)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == b2.STATUS_TIMEOUT
+    assert np.array_equal(x.host(), synth.vector_np(1, 1, n, np.float32))
+    ctx.reset()
     x = Guarded(synth.vector_np(1, 1, n, np.float32))
     b2.trsv(ctx, orc.ROW_MAJOR, orc.LOWER, orc.NO_TRANS, orc.NON_UNIT, n, a.t, n, x.t, 1)
     torch.cuda.synchronize()
@@ -281,3 +289,48 @@ def test_level2_determinism(b2, ctx, dtype):
         b2.trmv(ctx, orc.ROW_MAJOR, orc.LOWER, orc.TRANS, orc.NON_UNIT, n, a.t, n, gy.t, 1)
         outs.append(gy.host().copy())
     assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_workspace_query_is_enough(b2, dtype):
+    """A workspace of exactly b2_workspace_query(m, n, s) bytes serves every level-2 routine on an
+    m x n problem (the recommended default is only a default): a matrix of a few very long rows,
+    where the column splits of the row-dot kind must all be merged, and a triangular one."""
+    s = np.dtype(dtype).itemsize
+    tol = TOL[np.dtype(dtype)]
+    m, n = 6, 300000
+    small = b2.Context(workspace_bytes=b2.lib().b2_workspace_query(m, n, s))
+    small.reset()
+    a = synth.vector_np(41, 1, m * n, dtype)
+    ga = Guarded(a)
+    for trans in TRANSES:
+        lenx, leny = (n, m) if trans == orc.NO_TRANS else (m, n)
+        x, y = synth.vector_np(41, 2, lenx, dtype), synth.vector_np(41, 3, leny, dtype)
+        gx, gy = Guarded(x), Guarded(y)
+        b2.gemv(small, orc.ROW_MAJOR, trans, m, n, 1.25, ga.t, n, gx.t, 1, 0.5, gy.t, 1)
+        oy = y.copy()
+        absterms = orc.gemv(orc.ROW_MAJOR, trans, m, n, dtype(1.25), a, n, x, 1, dtype(0.5), oy, 1)
+        assert_close(gy.host(), oy, absterms, dtype, f"gemv trans={trans} on the queried workspace")
+        gy.check_guards()
+    k = 2100
+    tri = Guarded(synth.matrix_np(41, 4, k, k, k, dtype, tri_n=k).ravel())
+    small = b2.Context(workspace_bytes=b2.lib().b2_workspace_query(k, k, s))
+    small.reset()
+    v = synth.vector_np(41, 5, k, dtype)
+    gv, gy = Guarded(v), Guarded(v.copy())
+    b2.symv(small, orc.ROW_MAJOR, orc.LOWER, k, 1.25, tri.t, k, gv.t, 1, 0.5, gy.t, 1)
+    oy = v.copy()
+    absterms = orc.symv(orc.ROW_MAJOR, orc.LOWER, k, dtype(1.25), tri.host(), k, v, 1, dtype(0.5), oy, 1)
+    assert_close(gy.host(), oy, absterms, dtype, "symv on the queried workspace")
+    for trans in TRANSES:
+        gx = Guarded(v)
+        b2.trmv(small, orc.ROW_MAJOR, orc.UPPER, trans, orc.NON_UNIT, k, tri.t, k, gx.t, 1)
+        ox = v.copy()
+        absterms = orc.trmv(orc.ROW_MAJOR, orc.UPPER, trans, orc.NON_UNIT, k, tri.host(), k, ox, 1)
+        assert_close(gx.host(), ox, absterms, dtype, "trmv on the queried workspace")
+        gx = Guarded(v)
+        b2.trsv(small, orc.ROW_MAJOR, orc.UPPER, trans, orc.NON_UNIT, k, tri.t, k, gx.t, 1)
+        assert small.device_status() == 0
+        resid, scale = orc.trsv_residual(orc.ROW_MAJOR, orc.UPPER, trans, orc.NON_UNIT, k, tri.host(), k, v, 1,
+                                         gx.host(), 1)
+        assert np.all(resid <= tol * scale), "trsv on the queried workspace"
