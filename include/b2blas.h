@@ -77,7 +77,7 @@ typedef struct b2_ctx {
 } b2_ctx;
 
 size_t b2_workspace_min_bytes(void); /* control block + level-1 partials                   */
-/* Recommended size (64 MiB): a default, not a bound.  It serves every call on matrices up to
+/* Recommended size (256 MiB): a default, not a bound.  It serves every call on matrices up to
  * 32768 x 32768 and vectors of any length without B2_STATUS_WORKSPACE_TOO_SMALL; the exact
  * need of one call is b2_workspace_query's. */
 size_t b2_workspace_bytes(void);

@@ -15,6 +15,10 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobTrsvPrefetchBytes */ 48 << 20,
     /* kKnobTrsvFront       */ 2,
     /* kKnobTrsvCluster     */ 0,
+    /* kKnobTrsvHelpNear    */ 12,
+    /* kKnobTrsvHelpChunk   */ 8,
+    /* kKnobTrsvOwners      */ 48,
+    /* kKnobTrsvPmFrom      */ 10,
 };
 
 unsigned long long g_launch_count = 0;
@@ -38,16 +42,22 @@ int sm_count() {
 extern "C" {
 
 size_t b2_workspace_min_bytes(void) { return b2::kCtlBytes + 64 * 1024; }
-size_t b2_workspace_bytes(void) { return (size_t)64 << 20; }
+size_t b2_workspace_bytes(void) { return (size_t)256 << 20; }
 
 size_t b2_workspace_query(int64_t m, int64_t n, size_t elem_bytes) {
   if (m < 0 || n < 0 || (elem_bytes != 4 && elem_bytes != 8)) return 0;
   // level 1: one partial per block of the reduction grid; level 2 with every split merged: one
-  // row of partials per output vector; trsv: one or two tagged 64-bit words per unknown
-  const size_t vec = (size_t)(m > n ? m : n);
+  // row of partials per output vector; symv, whose blocks produce row sums and column sums at
+  // once: one row of partials per column tile of 32 packs; trsv: one or two
+  // tagged 64-bit words per unknown
+  const size_t vec = (size_t)(m > n ? m : n), sq = (size_t)(m < n ? m : n);
+  const size_t tile_cols = 32 * (16 / elem_bytes);
   const size_t level2 = ((size_t)m + (size_t)n) * elem_bytes + 1024;
+  const size_t symv = ((sq + tile_cols - 1) / tile_cols + 1) * sq * elem_bytes + 1024;
   const size_t trsv = vec * 8 * (elem_bytes / 4);
-  return b2_workspace_min_bytes() + (level2 > trsv ? level2 : trsv);
+  size_t need = level2 > trsv ? level2 : trsv;
+  if (symv > need) need = symv;
+  return b2_workspace_min_bytes() + need;
 }
 
 int b2_workspace_reset(const b2_ctx* ctx) {

@@ -410,8 +410,10 @@ static int l2_launch_shape(const Launch& l, L2Args<T> args, int64_t rows_per_cta
       args.colpart = reinterpret_cast<T*>(l.scratch + row_bytes);
       break;
     }
+    // (a block of a column-sum kind walks exactly S::NCT column tiles -- their sums sit in its
+    // registers -- so only its row band can grow; a row-dot kind merges column splits)
     bool changed = false;
-    if (K::ROWOUT && ctiles_per_cta < args.nct) ctiles_per_cta *= 2, changed = true;
+    if (K::ROWOUT && !K::COLOUT && ctiles_per_cta < args.nct) ctiles_per_cta *= 2, changed = true;
     if (ctiles_per_cta > args.nct) ctiles_per_cta = args.nct;
     if (K::COLOUT && rows_per_cta < args.rows) rows_per_cta *= 2, changed = true;
     if (!changed) return B2_STATUS_WORKSPACE_TOO_SMALL;

@@ -217,15 +217,21 @@ def test_trsv_bounded_wait_reports_timeout(b2):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
-@pytest.mark.parametrize("front,cluster", [(0, 0), (2, 0), (2, 2)])
-def test_trsv_every_kernel_choice(b2, ctx, dtype, front, cluster):
+@pytest.mark.parametrize("front,cluster,near,chunk", [(0, 0, 12, 8), (2, 0, 0, 8), (2, 2, 0, 8), (2, 0, 4, 2),
+                                                      (2, 2, 4, 2), (2, 0, 5, 4)])
+def test_trsv_every_kernel_choice(b2, ctx, dtype, front, cluster, near, chunk):
     """trsv has three code paths (block-row kernel; sub-block kernel block by block, which
-    premultiplies the last tile; sub-block kernel in clusters).  The defaults pick one per
-    precision and view; here each is forced for every view, on sizes with a ragged last block
-    and more block rows than one cluster holds."""
-    old = b2.get_tuning(b2.KNOB_TRSV_FRONT), b2.get_tuning(b2.KNOB_TRSV_CLUSTER)
+    premultiplies the last tile; sub-block kernel in clusters), and the sub-block kernel runs with
+    or without helper blocks that take the far tiles of long rows.  The defaults pick one per
+    precision, view and size; here each is forced for every view, on sizes with a ragged last
+    block and more block rows than one cluster holds, with helper units small enough that these
+    sizes have several per row."""
+    old = (b2.get_tuning(b2.KNOB_TRSV_FRONT), b2.get_tuning(b2.KNOB_TRSV_CLUSTER),
+           b2.get_tuning(b2.KNOB_TRSV_HELP_NEAR), b2.get_tuning(b2.KNOB_TRSV_HELP_CHUNK))
     b2.set_tuning(b2.KNOB_TRSV_FRONT, front)
     b2.set_tuning(b2.KNOB_TRSV_CLUSTER, cluster)
+    b2.set_tuning(b2.KNOB_TRSV_HELP_NEAR, near)
+    b2.set_tuning(b2.KNOB_TRSV_HELP_CHUNK, chunk)
     try:
         tol = TOL[np.dtype(dtype)]
         for n in (130, 1100, 2052):
@@ -242,6 +248,8 @@ def test_trsv_every_kernel_choice(b2, ctx, dtype, front, cluster):
     finally:
         b2.set_tuning(b2.KNOB_TRSV_FRONT, old[0])
         b2.set_tuning(b2.KNOB_TRSV_CLUSTER, old[1])
+        b2.set_tuning(b2.KNOB_TRSV_HELP_NEAR, old[2])
+        b2.set_tuning(b2.KNOB_TRSV_HELP_CHUNK, old[3])
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
