@@ -19,6 +19,7 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobTrsvHelpChunk   */ 8,
     /* kKnobTrsvOwners      */ 48,
     /* kKnobTrsvPmFrom      */ 10,
+    /* kKnobTriTile         */ 1,
 };
 
 unsigned long long g_launch_count = 0;

@@ -217,6 +217,7 @@ enum Knob {
   kKnobTrsvHelpNear = 11,      // tiles next to the diagonal an owner block keeps at least (0: no helper blocks)
   kKnobTrsvHelpChunk = 12,     // tiles per helper unit (even)
   kKnobTrsvOwners = 13,        // blocks that own rows when helpers run (the rest of the SMs help)
+  kKnobTriTile = 15,           // symv / trmv on aligned matrices: 1 = register-tile kernel, 0 = general tile kernel
   kKnobTrsvPmFrom = 14,        // first block row whose last tile is premultiplied by the inverse diagonal block
   kKnobCount = 16
 };

@@ -7,6 +7,7 @@
 //          written over x by the finalize kernel, after every block has finished reading x.
 #pragma once
 #include "level2.cuh"
+#include "tri_tile.cuh"
 
 namespace b2 {
 
@@ -56,6 +57,14 @@ static int symv_impl(const b2_ctx* ctx, int order, int uplo, int64_t n, T alpha,
   args.incy = incy;
   // the stored triangle as it sits in the row-major view of the buffer
   const bool upper = (order == B2_ROW_MAJOR) == (uplo == B2_UPPER);
+  if (knob(kKnobTriTile)) {  // 16-byte aligned matrices: the register-tile kernel
+    bool handled = false;
+    const int st = upper ? tt::tri_tile_run<T, true, true, TRI_UPPER, false, true>(l, a, lda, n, args.xc, incx, alpha, beta,
+                                                                                  args.y, incy, &handled)
+                         : tt::tri_tile_run<T, true, true, TRI_LOWER, false, true>(l, a, lda, n, args.xc, incx, alpha, beta,
+                                                                                  args.y, incy, &handled);
+    if (handled) return st;
+  }
   const L2Plan plan = plan_tri(args);
   if (upper) return l2_dispatch<T, Kind<true, true, TRI_UPPER, false, true>, false>(l, args, plan, false);
   return l2_dispatch<T, Kind<true, true, TRI_LOWER, false, true>, false>(l, args, plan, false);
@@ -63,6 +72,15 @@ static int symv_impl(const b2_ctx* ctx, int order, int uplo, int64_t n, T alpha,
 
 template <typename T, bool ROW, int TRI>
 static int trmv_kind(const Launch& l, const L2Args<T>& args, bool unit) {
+  if (knob(kKnobTriTile)) {  // 16-byte aligned matrices: the register-tile kernel
+    bool handled = false;
+    const int st =
+        unit ? tt::tri_tile_run<T, ROW, !ROW, TRI, true, false>(l, args.a, args.lda, args.rows, args.xc, args.incxc, T(1), T(0),
+                                                               args.y, args.incy, &handled)
+             : tt::tri_tile_run<T, ROW, !ROW, TRI, false, false>(l, args.a, args.lda, args.rows, args.xc, args.incxc, T(1), T(0),
+                                                                args.y, args.incy, &handled);
+    if (handled) return st;
+  }
   const L2Plan plan = ROW ? plan_rowout(args, false) : plan_colout(args, false, knob(kKnobTriRows));
   if (unit) return l2_dispatch<T, Kind<ROW, !ROW, TRI, true, false>, false>(l, args, plan, false);
   return l2_dispatch<T, Kind<ROW, !ROW, TRI, false, false>, false>(l, args, plan, false);

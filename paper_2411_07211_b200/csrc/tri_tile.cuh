@@ -1,0 +1,474 @@
+// symv and trmv on 16-byte aligned matrices: tile kernel with a shared-memory ring (Section 6.2.2, "Triangular
+// Matrix": the same loop nest as gemv over a triangular iteration space, bounds rounded to the
+// blocking factor so that full tiles run unmasked and only the tiles on the diagonal are masked).
+//
+// The canonical row-major view is cut into tiles of 128 rows x 32 packs (128 floats / 64 doubles).
+// A 256-thread block is a 16 x 16 grid; thread (rg, cg) holds rows 8*rg .. 8*rg+7 and the two
+// packs cg and cg + 16 of each (a half-warp covers 256 contiguous bytes of a row); the tile reaches
+// the thread through asynchronous copies into shared memory, several half tiles ahead (see the
+// kernel).  One pass over a tile serves
+//   row sums  (ROW): sum_j A_ij x_j, kept in 8 registers while the block walks ALONG a block row and
+//                    reduced over the 16 lanes of a row group once per unit, and / or
+//   column sums (COL): sum_i A_ij x_i, per tile: one exchange between the two half-warps, then one
+//                    store per warp into shared memory (no block-wide barrier per tile).
+// symv uses both on the stored triangle (each element loaded once, used twice; the diagonal only
+// in the row sum); trmv uses one of them with the diagonal taken as 1 for diag = unit.  A kind
+// that has only column sums walks DOWN a block column instead, with the column sums in registers.
+// Units (a few consecutive tiles) write partials to the workspace; tri_tile_finalize adds them in
+// a fixed order, so results are bit-reproducible, and writes y (trmv: x, after every block has
+// read it).
+#pragma once
+
+#include "level2.cuh"
+
+namespace b2 {
+namespace tt {
+
+// (measured: wider, flatter tiles -- 64 x 256 or 32 x 512 floats -- are slower here, they waste
+// more of the tiles that the diagonal cuts and make the units coarser)
+constexpr int kNR = 8;         // rows of a tile a thread holds
+constexpr int kNP = 2;         // packs of each row a thread holds (16 lanes side by side, kNP groups of them)
+constexpr int kTR = 16 * kNR;  // tile rows
+constexpr int kUnitMax = 4;    // tiles per unit at most (1, 2 or 4)
+constexpr int kRing = 3;      // tiles (64 KB each) in the shared-memory ring
+constexpr int kMaxMajor = 2048;  // block rows (or column tiles) the unit table can hold
+
+// Elements of the queue of x values: one slot per unit that can be in flight (kRing / unit + 2
+// units of `unit` tiles each), sized for the worst unit length.
+template <typename T, bool WALK_ROWS, bool ROWS_OF_X>
+__host__ __device__ constexpr int kSlotElems() {
+  constexpr int TC = 16 * kNP * VecLen<T>::value;
+  // along the walking direction a slot holds unit * tile extent values, across it one tile extent
+  constexpr int ext = ROWS_OF_X ? kTR : TC;
+  constexpr bool along = ROWS_OF_X != WALK_ROWS;
+  int worst = 0;
+  for (int unit = 1; unit <= kUnitMax; unit *= 2) {
+    const int need = (kRing / unit + 2) * (along ? unit : 1) * ext;
+    worst = need > worst ? need : worst;
+  }
+  return worst;
+}
+
+template <typename T>
+struct TileArgs {
+  const T* a;
+  int64_t lda, n;
+  const T* x;  // base per vec_base()
+  int64_t incx;
+  T* rowpart;  // [groups][n]: ROW kinds, one row of partials per column group (ROW && COL: per unit column group)
+  T* colpart;  // [groups][n]: COL kinds, one row of partials per block row (row walk) or row group (column walk)
+  int nbr, nct;  // block rows, column tiles
+  int unit;      // tiles per unit
+  int ngroups;   // units per block row (row walk) / per block column (column walk)
+  T alpha, beta;
+  T* y;
+  int64_t incy;
+  int prefix[kMaxMajor + 1];  // units before block row (column tile) i; the last entry is their total
+};
+
+// First and last column tile of block row I that meets the triangle.
+template <int TRI, int TC>
+__host__ __device__ __forceinline__ void row_range(int I, int64_t n, int nct, int* jlo, int* jhi) {
+  const int64_t r0 = (int64_t)I * kTR, r1 = (r0 + kTR < n ? r0 + kTR : n) - 1;
+  *jlo = TRI == TRI_UPPER ? (int)(r0 / TC) : 0;
+  *jhi = TRI == TRI_LOWER ? (int)(r1 / TC) : nct - 1;
+}
+// First and last block row of column tile J that meets the triangle.
+template <int TRI, int TC>
+__host__ __device__ __forceinline__ void col_range(int J, int64_t n, int nbr, int* ilo, int* ihi) {
+  const int64_t c0 = (int64_t)J * TC, c1 = (c0 + TC < n ? c0 + TC : n) - 1;
+  *ilo = TRI == TRI_LOWER ? (int)(c0 / kTR) : 0;
+  *ihi = TRI == TRI_UPPER ? (int)(c1 / kTR) : nbr - 1;
+}
+
+// Asynchronous 16-byte copy global -> shared memory of `bytes` (0 .. 16) bytes, the rest of the
+// 16 zero-filled; element-sized copies for the vectors (bytes = 0: a zero).
+__device__ __forceinline__ void cp_async16_full(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, int bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src),
+               "r"(bytes)
+               : "memory");
+}
+template <int N>
+__device__ __forceinline__ void cp_async_elem(void* dst, const void* src, bool valid) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src),
+               "n"(N), "r"(valid ? N : 0)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// Persistent blocks (one per SM).  Block b takes the units b, b + gridDim, ... of the dense unit
+// list and streams their tiles through a ring of kRing tiles in shared memory filled by
+// asynchronous copies: every thread copies exactly the 16 packs it will later read itself, so the
+// ring needs no barrier -- only the per-thread wait for its own copies -- and the copies of the
+// next kRing - 1 tiles (also those of the block's next units) are in flight while a tile is
+// multiplied.  Edge tiles use the same copies with a byte count that zero-fills what lies outside
+// the matrix.  The x values of a unit travel the same way.
+template <typename T, bool ROW, bool COL, int TRI, bool UNIT, bool SYM>
+__global__ void __launch_bounds__(kThreads, 1) tri_tile_kernel(const TileArgs<T> p) {
+  constexpr int V = VecLen<T>::value, TC = 16 * kNP * V, NR = kNR, HR = NR / 2, NP = kNP, TP = NR * NP;
+  constexpr bool WALK_ROWS = ROW;  // column-sum-only kinds walk down a block column
+  constexpr int XCU = WALK_ROWS ? kUnitMax * TC : TC;  // most column values a unit needs
+  using P = Pack<T, V>;
+  grid_dep_launch();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint4* ring = reinterpret_cast<uint4*>(smem_raw);             // [kRing][TP][kThreads] packs
+  T* xr_q = reinterpret_cast<T*>(ring + kRing * TP * kThreads);  // [slots] row values of the units in flight
+  constexpr int XRQ = COL ? kSlotElems<T, WALK_ROWS, true>() : 0, XCQ = ROW ? kSlotElems<T, WALK_ROWS, false>() : 0;
+  T* xc_q = xr_q + XRQ;  // [slots] column values
+  T* cbuf = xc_q + XCQ;  // [kWarps][XCU] column sums of the warps
+
+  const int ct = (int)threadIdx.x, warp = ct >> 5, lane = ct & 31;
+  const int rg = ct >> 4, cg = ct & 15;
+  const int nmajor = WALK_ROWS ? p.nbr : p.nct;
+  const int nunits = p.prefix[nmajor];
+  const int nslots = kRing / p.unit + 2;  // units that can be between the two cursors, plus one
+  const int xr_stride = WALK_ROWS ? kTR : p.unit * kTR, xc_stride = WALK_ROWS ? p.unit * TC : TC;
+  const int64_t row_step = p.lda;                              // elements between a thread's rows
+  const int64_t thread_off = (int64_t)(rg * HR) * p.lda + V * cg;  // this thread's first pack inside a half tile
+  const int64_t half_step = (int64_t)(kTR / 2) * p.lda;
+
+  // A cursor walks the block's sequence of tiles; the units come in increasing order, so the row
+  // (column) a unit belongs to is found by moving forward through the unit table.
+  struct Cursor {
+    int u, major, g, t0, t1, t, slot;
+    bool valid;
+  };
+  auto open_unit = [&](Cursor& c) {
+    c.valid = c.u < nunits;
+    if (!c.valid) return;
+    while (p.prefix[c.major + 1] <= c.u) ++c.major;
+    c.g = c.u - p.prefix[c.major];
+    int rl, rh;
+    if (WALK_ROWS) row_range<TRI, TC>(c.major, p.n, p.nct, &rl, &rh);
+    else col_range<TRI, TC>(c.major, p.n, p.nbr, &rl, &rh);
+    c.t0 = max(rl, (rl / p.unit + c.g) * p.unit);
+    c.t1 = min(rh, (rl / p.unit + c.g) * p.unit + p.unit - 1);
+    c.t = c.t0;
+  };
+  auto advance = [&](Cursor& c) {
+    if (++c.t <= c.t1) return;
+    c.u += (int)gridDim.x;
+    c.slot = c.slot + 1 == nslots ? 0 : c.slot + 1;
+    open_unit(c);
+  };
+
+  Cursor prod, cons;
+  prod.u = cons.u = (int)blockIdx.x;
+  prod.slot = cons.slot = 0;
+  prod.major = cons.major = 0;
+  open_unit(prod);
+  open_unit(cons);
+  int pstage = 0, cstage = 0;
+
+  // one producer step: the copies of the next tile (and, with a unit's first one, of its x values)
+  auto produce = [&]() {
+    if (prod.valid) {
+      const int I = WALK_ROWS ? prod.major : prod.t, J = WALK_ROWS ? prod.t : prod.major;
+      const int64_t r0 = (int64_t)I * kTR, c0 = (int64_t)J * TC;
+      if (prod.t == prod.t0) {
+        const int64_t rb = (int64_t)(WALK_ROWS ? I : prod.t0) * kTR, cb = (int64_t)(WALK_ROWS ? prod.t0 : J) * TC;
+        const int nrv = (WALK_ROWS ? 1 : prod.t1 - prod.t0 + 1) * kTR, ncv = (WALK_ROWS ? prod.t1 - prod.t0 + 1 : 1) * TC;
+        if (COL)
+          for (int t = ct; t < nrv; t += kThreads) {
+            const bool ok = rb + t < p.n;
+            cp_async_elem<sizeof(T)>(xr_q + prod.slot * xr_stride + t, p.x + (ok ? (rb + t) * p.incx : 0), ok);
+          }
+        if (ROW)
+          for (int t = ct; t < ncv; t += kThreads) {
+            const bool ok = cb + t < p.n;
+            cp_async_elem<sizeof(T)>(xc_q + prod.slot * xc_stride + t, p.x + (ok ? (cb + t) * p.incx : 0), ok);
+          }
+      }
+      uint4* dst = ring + (size_t)pstage * TP * kThreads + ct;
+      const T* src = p.a + r0 * p.lda + c0 + thread_off;
+      if (r0 + kTR <= p.n && c0 + TC <= p.n) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int a = 0; a < HR; ++a)
+#pragma unroll
+            for (int hb = 0; hb < NP; ++hb)
+              cp_async16_full(dst + ((h * HR + a) * NP + hb) * kThreads, src + h * half_step + a * row_step + hb * 16 * V);
+      } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int a = 0; a < HR; ++a) {
+            const int64_t r = r0 + h * (kTR / 2) + rg * HR + a;
+#pragma unroll
+            for (int hb = 0; hb < NP; ++hb) {
+              const int64_t left = (p.n - (c0 + V * cg + hb * 16 * V)) * (int64_t)sizeof(T);
+              const int bytes = (r < p.n && left > 0) ? (int)(left < 16 ? left : 16) : 0;
+              cp_async16(dst + ((h * HR + a) * NP + hb) * kThreads,
+                         bytes ? src + h * half_step + a * row_step + hb * 16 * V : p.a, bytes);
+            }
+          }
+      }
+      advance(prod);
+    }
+    cp_async_commit();  // (an empty group when the sequence has ended: the group count stays uniform)
+    pstage = pstage + 1 == kRing ? 0 : pstage + 1;
+  };
+
+  T racc[NR], cacc[NP][V];
+#pragma unroll
+  for (int a = 0; a < NR; ++a) racc[a] = T(0);
+#pragma unroll
+  for (int hb = 0; hb < NP; ++hb)
+#pragma unroll
+    for (int e = 0; e < V; ++e) cacc[hb][e] = T(0);
+
+#pragma unroll 1
+  for (int s = 0; s < kRing - 1; ++s) produce();
+#pragma unroll 1
+  while (cons.valid) {
+    produce();
+    cp_async_wait<kRing - 1>();  // this thread's copies of the oldest tile in flight have landed
+    const int I = WALK_ROWS ? cons.major : cons.t, J = WALK_ROWS ? cons.t : cons.major;
+    const int I0 = WALK_ROWS ? I : cons.t0, J0 = WALK_ROWS ? cons.t0 : J;
+    if (cons.t == cons.t0) __syncthreads();  // the unit's x values came from other threads' copies
+    const int64_t r0 = (int64_t)I * kTR, c0 = (int64_t)J * TC;
+    const uint4* src = ring + (size_t)cstage * TP * kThreads + ct;
+    cstage = cstage + 1 == kRing ? 0 : cstage + 1;
+    T xc[NP][V];
+    if (ROW) {
+      const T* xs = xc_q + cons.slot * xc_stride + (J - J0) * TC + V * cg;
+#pragma unroll
+      for (int hb = 0; hb < NP; ++hb) {
+        const P pk = *reinterpret_cast<const P*>(xs + hb * 16 * V);
+#pragma unroll
+        for (int e = 0; e < V; ++e) xc[hb][e] = pk.v[e];
+      }
+    }
+    // no element of the tile on or beyond the diagonal: nothing to mask (what lies outside the
+    // matrix arrived as zeros)
+    const bool inside = TRI == TRI_FULL || (TRI == TRI_LOWER ? c0 + TC - 1 < r0 : c0 > r0 + kTR - 1);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {  // the two halves of the tile (rows 0 .. 63, 64 .. 127)
+      T m[HR][NP][V];
+#pragma unroll
+      for (int a = 0; a < HR; ++a)
+#pragma unroll
+        for (int hb = 0; hb < NP; ++hb) {
+          const uint4 raw = src[((h * HR + a) * NP + hb) * kThreads];
+          const P pk = *reinterpret_cast<const P*>(&raw);
+#pragma unroll
+          for (int e = 0; e < V; ++e) m[a][hb][e] = pk.v[e];
+        }
+      T xr[HR];
+      if (COL) {
+        const T* xs = xr_q + cons.slot * xr_stride + (I - I0) * kTR + h * (kTR / 2) + rg * HR;
+#pragma unroll
+        for (int a = 0; a < HR; ++a) xr[a] = xs[a];
+      }
+      if (inside) {
+#pragma unroll
+        for (int a = 0; a < HR; ++a)
+#pragma unroll
+          for (int hb = 0; hb < NP; ++hb)
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+              if (ROW) racc[h * HR + a] = m[a][hb][e] * xc[hb][e] + racc[h * HR + a];
+              if (COL) cacc[hb][e] = m[a][hb][e] * xr[a] + cacc[hb][e];
+            }
+      } else {
+        // a tile on the diagonal: d = (column of the element) - (row of the element)
+        const int dbase = (int)(c0 - r0) - h * (kTR / 2) + V * cg - rg * HR;
+        const int nrows = (int)min((int64_t)(kTR / 2), p.n - r0 - h * (kTR / 2));
+#pragma unroll
+        for (int a = 0; a < HR; ++a)
+#pragma unroll
+          for (int hb = 0; hb < NP; ++hb)
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+              const int d = dbase + hb * 16 * V + e - a;
+              const bool in_tri = TRI == TRI_LOWER ? d <= 0 : d >= 0;
+              T v = in_tri ? m[a][hb][e] : T(0);
+              if (UNIT && d == 0) v = (rg * HR + a < nrows) ? T(1) : T(0);
+              if (ROW) racc[h * HR + a] = v * xc[hb][e] + racc[h * HR + a];
+              if (COL) cacc[hb][e] = ((SYM && d == 0) ? T(0) : v) * xr[a] + cacc[hb][e];
+            }
+      }
+    }
+    const bool unit_done = cons.t == cons.t1;
+    if (COL && (WALK_ROWS || unit_done)) {
+      // column sums: the two row groups of the warp, then shared memory; along a block row per tile
+#pragma unroll
+      for (int hb = 0; hb < NP; ++hb) {
+        P pk;
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          pk.v[e] = cacc[hb][e] + shfl_xor(cacc[hb][e], 16);
+          cacc[hb][e] = T(0);
+        }
+        if (lane < 16) *reinterpret_cast<P*>(cbuf + warp * XCU + (J - J0) * TC + V * cg + hb * 16 * V) = pk;
+      }
+    }
+    if (unit_done) {
+      const int64_t r_base = (int64_t)I0 * kTR, c_base = (int64_t)J0 * TC;
+      if (ROW) {  // 8 row sums over the 16 lanes of a row group: lanes 2v and 2v + 1 end up with value v
+        const T s = multi_group_sum<16, NR>(racc, lane);
+        constexpr int LPV = 16 / NR;  // lanes that end up with the same value
+        const int v = cg / LPV;
+        const int64_t i = r_base + (v / HR) * (kTR / 2) + rg * HR + v % HR;
+        if (cg % LPV == 0 && i < p.n) p.rowpart[(int64_t)cons.g * p.n + i] = s;
+#pragma unroll
+        for (int a = 0; a < NR; ++a) racc[a] = T(0);
+      }
+      if (COL) {
+        const int ncols = (WALK_ROWS ? cons.t1 - cons.t0 + 1 : 1) * TC;
+        __syncthreads();
+        for (int t = ct; t < ncols; t += kThreads) {
+          if (c_base + t >= p.n) break;
+          T s = cbuf[t];
+#pragma unroll
+          for (int w = 1; w < kWarps; ++w) s += cbuf[w * XCU + t];
+          p.colpart[(int64_t)(WALK_ROWS ? cons.major : cons.g) * p.n + c_base + t] = s;
+        }
+        __syncthreads();  // cbuf is written again by the next unit
+      }
+    }
+    advance(cons);
+  }
+  cp_async_wait<0>();
+}
+
+// y_i = alpha * (row partials of i + column partials of i) + beta * y_i, the partials added in a
+// fixed order.  A block of 32 warps serves 32 consecutive outputs (one per lane, so every load is
+// a coalesced row segment of a partial array); warp w takes partials w, w + 32, ... -- a handful
+// of independent loads, all in flight at once -- and warp 0 adds the 32 sums in warp order.
+constexpr int kFinWarps = 32;
+template <typename T, bool ROW, bool COL, int TRI>
+__global__ void __launch_bounds__(kFinWarps * 32) tri_tile_finalize(const TileArgs<T> p) {
+  constexpr int V = VecLen<T>::value, TC = 16 * kNP * V;
+  constexpr bool WALK_ROWS = ROW;
+  __shared__ T part[kFinWarps][33];
+  grid_dep_wait();
+  const int w = (int)(threadIdx.x >> 5), lane = (int)(threadIdx.x & 31);
+  const int64_t i = (int64_t)blockIdx.x * 32 + lane;
+  T s = T(0);
+  if (i < p.n) {
+    int nrow = 0;
+    if (ROW) {  // the units of i's block row
+      int lo, hi;
+      row_range<TRI, TC>((int)(i / kTR), p.n, p.nct, &lo, &hi);
+      nrow = hi / p.unit - lo / p.unit + 1;
+    }
+    int clo = 0, ncol = 0;
+    if (COL) {
+      int lo, hi;
+      col_range<TRI, TC>((int)(i / TC), p.n, p.nbr, &lo, &hi);
+      // along block rows: one partial per block row that meets i's column tile; down block
+      // columns: one per unit of i's block column
+      clo = WALK_ROWS ? lo : 0;
+      ncol = WALK_ROWS ? hi - lo + 1 : hi / p.unit - lo / p.unit + 1;
+    }
+    T s0 = T(0), s1 = T(0), s2 = T(0), s3 = T(0);
+    auto fetch = [&](int k) -> T {
+      if (k >= nrow + ncol) return T(0);
+      return k < nrow ? __ldcg(p.rowpart + (int64_t)k * p.n + i) : __ldcg(p.colpart + (int64_t)(clo + k - nrow) * p.n + i);
+    };
+    for (int k = w; k < nrow + ncol; k += 4 * kFinWarps) {
+      const T v0 = fetch(k), v1 = fetch(k + kFinWarps), v2 = fetch(k + 2 * kFinWarps), v3 = fetch(k + 3 * kFinWarps);
+      s0 += v0, s1 += v1, s2 += v2, s3 += v3;
+    }
+    s = (s0 + s1) + (s2 + s3);
+  }
+  part[w][lane] = s;
+  __syncthreads();
+  if (w == 0 && i < p.n) {
+    T t = part[0][lane];
+#pragma unroll
+    for (int k = 1; k < kFinWarps; ++k) t += part[k][lane];
+    T* yp = p.y + i * p.incy;
+    *yp = p.beta != T(0) ? p.alpha * t + p.beta * *yp : p.alpha * t;
+  }
+}
+
+// Shared memory of the tile kernel: the ring, the queues of x values, the warps' column sums.
+template <typename T, bool ROW, bool COL>
+constexpr size_t tile_smem_bytes() {
+  constexpr int TC = 16 * kNP * VecLen<T>::value;
+  constexpr bool WALK_ROWS = ROW;
+  return (size_t)kRing * kNR * kNP * kThreads * 16 +
+         sizeof(T) * (size_t)((COL ? kSlotElems<T, WALK_ROWS, true>() : 0) + (ROW ? kSlotElems<T, WALK_ROWS, false>() : 0) +
+                              (COL ? kWarps * (WALK_ROWS ? kUnitMax * TC : TC) : 0));
+}
+
+// Launches both kernels.  *handled is false (nothing launched) when the matrix is not 16-byte
+// aligned, too large for the unit table, or the partials do not fit the workspace: the caller
+// then uses the general tile kernel.
+template <typename T, bool ROW, bool COL, int TRI, bool UNIT, bool SYM>
+static int tri_tile_run(const Launch& l, const T* a, int64_t lda, int64_t n, const T* x, int64_t incx, T alpha, T beta,
+                        T* y, int64_t incy, bool* handled) {
+  constexpr int V = VecLen<T>::value, TC = 16 * kNP * V;
+  constexpr bool WALK_ROWS = ROW;
+  *handled = false;
+  if (!aligned_to(a, 16) || lda % V != 0) return B2_STATUS_OK;
+  const int64_t nbr = (n + kTR - 1) / kTR, nct = (n + TC - 1) / TC;
+  if ((WALK_ROWS ? nbr : nct) > kMaxMajor) return B2_STATUS_OK;
+  TileArgs<T> args = {};
+  args.a = a;
+  args.lda = lda;
+  args.n = n;
+  args.x = x;
+  args.incx = incx;
+  args.nbr = (int)nbr;
+  args.nct = (int)nct;
+  // a few thousand units keep the tail short; beyond that, longer units mean fewer partials
+  const int64_t tiles = nbr * nct / 2;
+  const int64_t want = tiles / ((int64_t)sm_count() * 16);
+  args.unit = (want >= 4 && kUnitMax >= 4) ? 4 : (want >= 2 && kUnitMax >= 2) ? 2 : 1;
+  const int nmajor = WALK_ROWS ? args.nbr : args.nct;
+  int ngroups = 0;
+  for (int i = 0; i < nmajor; ++i) {
+    int lo, hi;
+    if (WALK_ROWS) row_range<TRI, TC>(i, n, args.nct, &lo, &hi);
+    else col_range<TRI, TC>(i, n, args.nbr, &lo, &hi);
+    const int ng = hi / args.unit - lo / args.unit + 1;
+    args.prefix[i + 1] = args.prefix[i] + ng;
+    ngroups = ng > ngroups ? ng : ngroups;
+  }
+  args.ngroups = ngroups;
+  const size_t row_bytes = ROW ? ((size_t)ngroups * n * sizeof(T) + 255) / 256 * 256 : 0;
+  const size_t col_bytes = COL ? (size_t)(WALK_ROWS ? args.nbr : ngroups) * n * sizeof(T) : 0;
+  if (row_bytes + col_bytes > l.scratch_bytes) return B2_STATUS_OK;
+  args.rowpart = reinterpret_cast<T*>(l.scratch);
+  args.colpart = reinterpret_cast<T*>(l.scratch + row_bytes);
+  args.alpha = alpha;
+  args.beta = beta;
+  args.y = y;
+  args.incy = incy;
+  constexpr size_t smem = tile_smem_bytes<T, ROW, COL>();
+  auto kern = tri_tile_kernel<T, ROW, COL, TRI, UNIT, SYM>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return B2_STATUS_OK;
+  }
+  *handled = true;
+  const int nunits = args.prefix[nmajor];
+  const int grid = nunits < sm_count() ? nunits : sm_count();
+  kern<<<grid, kThreads, smem, l.stream>>>(args);
+  if (int st = check_launch()) return st;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((n + 31) / 32));
+  cfg.blockDim = dim3(kFinWarps * 32);
+  cfg.stream = l.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = knob(kKnobUsePdl) ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, tri_tile_finalize<T, ROW, COL, TRI>, args);
+  return check_launch();
+}
+
+}  // namespace tt
+}  // namespace b2
