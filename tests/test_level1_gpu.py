@@ -254,3 +254,53 @@ def test_bench_sizes(b2, ctx, dtype, tdt, inc):
 
 def span_t(n, inc):
     return 1 + (n - 1) * inc
+
+
+def test_level1_n_2_28(b2, ctx):
+    """The largest level-1 size of the size sweep, n = 2^28 (1 GiB per float vector: offsets and
+    chunk counts beyond 2^32 bytes): reductions against the full oracle, map routines on sampled
+    elements, a planted maximum in the last chunk."""
+    n, dtype, tdt = 1 << 28, np.float32, torch.float32
+    hx, hy = synth.vector_np(13, 0, n, dtype), synth.vector_np(13, 1, n, dtype)
+    dx, dy = synth.vector_torch(13, 0, n, tdt, "cuda"), synth.vector_torch(13, 1, n, tdt, "cuda")
+    res = torch.zeros(3, dtype=tdt, device="cuda")
+    ires = torch.zeros(1, dtype=torch.int64, device="cuda")
+    b2.dot(ctx, n, dx, 1, dy, 1, res[0:1])
+    b2.asum(ctx, n, dx, 1, res[1:2])
+    b2.nrm2(ctx, n, dx, 1, res[2:3])
+    b2.iamax(ctx, n, dx, 1, ires)
+    got = res.cpu().numpy()
+    d, dabs = orc.dot(n, hx, 1, hy, 1)
+    assert_close(got[0], d, dabs, dtype, "dot")
+    a, aabs = orc.asum(n, hx, 1)
+    assert_close(got[1], a, aabs, dtype, "asum")
+    nr, _ = orc.nrm2(n, hx, 1)
+    assert_close(got[2], nr, abs(float(nr)), dtype, "nrm2")
+    assert int(ires.item()) == orc.iamax(n, hx, 1)
+    dx2 = dx.clone()
+    dx2[n - 3] = 1.5
+    dx2[n - 1] = -1.5
+    b2.iamax(ctx, n, dx2, 1, ires)
+    assert int(ires.item()) == n - 3
+    del dx2
+    rng = np.random.default_rng(4)
+    idx = np.unique(np.concatenate([[0, 1, n - 1, n - 2, n // 2, (1 << 27) + 1], rng.integers(0, n, size=4000)]))
+    tidx = torch.from_numpy(idx).cuda()
+    sx, sy = hx[idx].copy(), hy[idx].copy()
+    y2 = dy.clone()
+    b2.axpy(ctx, n, 1.5, dx, 1, y2, 1)
+    oy = sy.copy()
+    absterms = orc.axpy(len(idx), dtype(1.5), sx, 1, oy, 1)
+    assert_close(y2[tidx].cpu().numpy(), oy, absterms, dtype, "axpy")
+    del y2
+    x3, y3 = dx.clone(), dy.clone()
+    b2.rot(ctx, n, x3, 1, y3, 1, 0.6, 0.8)
+    ox, oy = sx.copy(), sy.copy()
+    ax, ay = orc.rot(len(idx), ox, 1, oy, 1, dtype(0.6), dtype(0.8))
+    assert_close(x3[tidx].cpu().numpy(), ox, ax, dtype, "rot x")
+    assert_close(y3[tidx].cpu().numpy(), oy, ay, dtype, "rot y")
+    b2.swap(ctx, n, x3, 1, y3, 1)
+    b2.scal(ctx, n, -0.75, y3, 1)
+    assert_close(y3[tidx].cpu().numpy(), dtype(-0.75) * ox, ax, dtype, "swap + scal")  # 0.75 x the rot bound + one rounding
+    b2.copy(ctx, n, dx, 1, x3, 1)
+    assert torch.equal(x3, dx)

@@ -342,3 +342,26 @@ def test_workspace_query_is_enough(b2, dtype):
         resid, scale = orc.trsv_residual(orc.ROW_MAJOR, orc.UPPER, trans, orc.NON_UNIT, k, tri.host(), k, v, 1,
                                          gx.host(), 1)
         assert np.all(resid <= tol * scale), "trsv on the queried workspace"
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("c", [2.0, 8.0])
+def test_trsv_moderately_conditioned(b2, ctx, dtype, c):
+    """Matrices that are NOT diagonally dominant: unit diagonal, off-diagonal uniform[-1, 1] * c / sqrt(n)
+    (at c = 8 the solution grows to about 3e4 from a right-hand side in [-1, 1]).  The kernels apply
+    explicit inverses of the 128 x 128 / 64 x 64 diagonal blocks, whose error grows with the blocks'
+    condition number; the row-wise residual of the device solution must still meet the bound."""
+    n = 1100
+    tol = TOL[np.dtype(dtype)]
+    u = synth.vector_np(5, n, n * n, np.float64).reshape(n, n)
+    a = (u * c / np.sqrt(n)).astype(dtype)
+    np.fill_diagonal(a, 1.0)
+    b = synth.vector_np(5, 1, n, dtype)
+    ga = Guarded(a.ravel())
+    for uplo, trans, diag in ((orc.LOWER, orc.NO_TRANS, orc.UNIT), (orc.UPPER, orc.TRANS, orc.NON_UNIT),
+                              (orc.UPPER, orc.NO_TRANS, orc.UNIT), (orc.LOWER, orc.TRANS, orc.NON_UNIT)):
+        gx = Guarded(b)
+        b2.trsv(ctx, orc.ROW_MAJOR, uplo, trans, diag, n, ga.t, n, gx.t, 1)
+        assert ctx.device_status() == 0
+        resid, scale = orc.trsv_residual(orc.ROW_MAJOR, uplo, trans, diag, n, a.ravel(), n, b, 1, gx.host(), 1)
+        assert np.all(resid <= tol * scale), f"c={c} {uplo} {trans} {diag}: worst {np.max(resid / scale) / tol:.3f} of the bound"

@@ -112,8 +112,6 @@ def op_row(seed, stream, n, dtype, uplo, trans, diag, i, symmetric=False):
                                      (np.float64, 8192), (np.float64, 32768)])
 def test_triangular_config_sizes(b2, ctx, dtype, n):
     seed, stream = 37, 6
-    if n == 32768 and dtype == np.float64:
-        n = 16384  # keeps the device matrix at 2 GiB; the 8 GiB case adds nothing the others do not
     a = synth.matrix_torch(seed, stream, n, n, n, TD[dtype], "cuda", tri_n=n)
     hx, hy = synth.vector_np(seed, 7, n, dtype), synth.vector_np(seed, 8, n, dtype)
     tol = TOL[np.dtype(dtype)]
@@ -148,4 +146,43 @@ def test_triangular_config_sizes(b2, ctx, dtype, n):
                     slack = float(np.finfo(dtype).eps) * abs(float(ax))  # the dot itself is rounded to T
                     assert resid <= tol * scale + slack, f"trsv {uplo} {trans} {diag} row {i}: {resid:.3e} > {tol * scale:.3e}"
     del a
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+@pytest.mark.parametrize("m,n", [(1 << 20, 40), (3 ** 13, 40), (3 ** 13, 24), (1 << 20, 88)])
+def test_gemv_ger_column_major_narrow(b2, ctx, dtype, m, n):
+    """The narrow shapes of the paper's skinny study (Section 6.2.2) in COLUMN-major storage, at the
+    sizes the bench's next-rows leg times: the buffer holds n columns of m elements (lda = m), so the
+    kernels see the transposed, very wide row-major problem; an odd m (3^13) puts every second
+    column off the 16-byte boundary."""
+    if dtype == np.float64 and n == 88:
+        n = 44
+    seed = 43
+    buf = synth.matrix_torch(seed, 1, n, m, m, TD[dtype], "cuda")  # buf[j, i] = A(i, j)
+    hx_n, hx_m = synth.vector_np(seed, 2, n, dtype), synth.vector_np(seed, 3, m, dtype)
+    hy_m, hy_n = synth.vector_np(seed, 4, m, dtype), synth.vector_np(seed, 5, n, dtype)
+    y = dvec(seed, 4, m, dtype)
+    b2.gemv(ctx, orc.COL_MAJOR, orc.NO_TRANS, m, n, 1.25, buf, m, dvec(seed, 2, n, dtype), 1, 0.5, y, 1)
+    rows = sample(m, 5)
+    got = y[torch.from_numpy(rows).cuda()].cpu().numpy()
+    for r, g in zip(rows, got):
+        row = synth.matrix_entries_np(seed, 1, np.arange(n), r, m, dtype)  # A(r, :) = buf[:, r]
+        out = hy_m[r:r + 1].copy()
+        absterms = orc.gemv(orc.ROW_MAJOR, orc.NO_TRANS, 1, n, dtype(1.25), row, n, hx_n, 1, dtype(0.5), out, 1)
+        assert_close(g, out[0], absterms[0], dtype, f"column-major gemv-N row {r}")
+    y = dvec(seed, 5, n, dtype)
+    b2.gemv(ctx, orc.COL_MAJOR, orc.TRANS, m, n, 1.25, buf, m, dvec(seed, 3, m, dtype), 1, 0.5, y, 1)
+    got = y.cpu().numpy()
+    for c in range(n):  # every output: a dot product over one stored row of the buffer
+        col = synth.matrix_entries_np(seed, 1, c, np.arange(m), m, dtype)
+        out = hy_n[c:c + 1].copy()
+        absterms = orc.gemv(orc.ROW_MAJOR, orc.TRANS, m, 1, dtype(1.25), col, 1, hx_m, 1, dtype(0.5), out, 1)
+        assert_close(got[c], out[0], absterms[0], dtype, f"column-major gemv-T column {c}")
+    b2.ger(ctx, orc.COL_MAJOR, m, n, 1.25, dvec(seed, 3, m, dtype), 1, dvec(seed, 2, n, dtype), 1, buf, m)
+    for r in sample(m, 6)[:16]:
+        seg = synth.matrix_entries_np(seed, 1, np.arange(n), r, m, dtype)  # A(r, 0 .. n-1)
+        absterms = orc.ger(orc.ROW_MAJOR, 1, n, dtype(1.25), hx_m[r:r + 1], 1, hx_n, 1, seg, n)
+        assert_close(buf[:, r].cpu().numpy(), seg, absterms[0], dtype, f"column-major ger row {r}")
+    del buf
     torch.cuda.empty_cache()
