@@ -28,6 +28,7 @@ sys.path.insert(0, ROOT)
 MIB = 1 << 20
 ROW, COL, NOTR, TR, UP, LO, NONU, UNIT = 101, 102, 111, 112, 121, 122, 131, 132
 FALLBACK_PEAK_GBS = 6650.0
+NOMINAL_PEAK_GBS = 8000.0  # the vendor's spec-sheet HBM3e figure for this part (second denominator)
 
 
 def ncu_dram_bytes_per_launch():
@@ -349,6 +350,180 @@ def next_rows_leg(wl: GpuWorkload, steps: int, peak: float, only=None):
             "geomean_frac": geomean([r["frac"] for r in rows]), "variants": rows}
 
 
+def configs_leg(device, peak: float, reps: int, only=None):
+    """The size sweeps beside the headline set (not part of `value`): the 1 Mi-element float dot
+    product; the level-1 routines at n = 2^16 .. 2^28; gemv / ger at 4096^2, 16384^2, 2^20 x 64 and
+    64 x 2^20 with beta 0 and 0.5; symv / trmv / trsv at n = 1024, 8192, 32768.  Working sets below
+    the L2 size are timed twice and labelled: "hot" (the same buffers every call: L2-resident, NOT
+    an HBM figure) and "cold" (calls rotate through enough distinct buffers to exceed twice the L2
+    size); larger ones once, behind a sweep of L2 like the headline set.  Small calls are timed in
+    batches (one event pair around `reps` calls) because a single call is shorter than the timer's
+    resolution."""
+    import torch
+    from paper_2411_07211_b200 import binding as b2
+    from paper_2411_07211_b200 import synth
+    ctx = b2.Context(device)
+    ctx.reset()
+    l2 = int(torch.cuda.get_device_properties(device).L2_cache_size)
+    flush = torch.zeros(64 * MIB, dtype=torch.float32, device=device)
+    fres = torch.zeros(1, dtype=torch.float32, device=device)
+    tdt = {"f32": torch.float32, "f64": torch.float64}
+    rows = []
+
+    def batch_ms(call, nbuf, count):
+        """Median over 5 batches of `count` calls (buffer k % nbuf), per call."""
+        ts = []
+        for it in range(7):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for k in range(count):
+                call(k % nbuf)
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                ts.append(e0.elapsed_time(e1) / count)
+        ts.sort()
+        return ts[len(ts) // 2]
+
+    def swept_ms(call):
+        ts = []
+        for it in range(reps + 3):
+            b2.asum(ctx, flush.numel(), flush, 1, fres)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            call(0)
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                ts.append(e0.elapsed_time(e1))
+        ts.sort()
+        return ts[len(ts) // 2]
+
+    def emit(name, ms, touched, label):
+        gbs = touched / (ms * 1e-3) / 1e9
+        rows.append({"name": name, "l2": label, "us": round(ms * 1e3, 2), "gbs": round(gbs, 1),
+                     "frac": round(gbs / peak, 4), "frac_nominal": round(gbs / NOMINAL_PEAK_GBS, 4)})
+
+    def measure(name, make_call, ws_bytes, touched, max_sets=None):
+        """make_call(nbuf) -> call(k): the routine on buffer set k of nbuf."""
+        if only and not any(k in name for k in only.split(",")):
+            return
+        if ws_bytes < l2:
+            nbuf = max(2, -(-2 * l2 // ws_bytes) + 1)
+            if max_sets:
+                nbuf = min(nbuf, max_sets)
+            call = make_call(nbuf)
+            count = max(8, min(256, nbuf))
+            emit(name, batch_ms(call, 1, count), touched, "hot (L2-resident)")
+            label = "cold (rotating buffers > 2 x L2)" if nbuf * ws_bytes > 2 * l2 else "cold (rotating buffers, < 2 x L2)"
+            emit(name, batch_ms(call, nbuf, max(count, nbuf)), touched, label)
+        else:
+            emit(name, swept_ms(make_call(1)), touched, "cold (working set > L2, L2 swept before each call)")
+
+    # ---- level 1: config 1 (sdot, 1 Mi floats) is the n = 2^20 row of the sweep
+    for dt, s in (("f32", 4), ("f64", 8)):
+        pool = synth.vector_torch(0, 20, (768 * MIB) // s, tdt[dt], device)  # rotating sets are slices of this
+        for lg in (16, 20, 24, 28):
+            n = 1 << lg
+            for inc in (1, 2):
+                span = n * inc
+                if 2 * span > pool.numel():
+                    continue  # (2^28 doubles with increment 2 would need 8 GiB for two vectors)
+                res = torch.zeros(4, dtype=tdt[dt], device=device)
+                ires = torch.zeros(1, dtype=torch.int64, device=device)
+                for r, per_elem, nvec in (("axpy", 3, 2), ("scal", 2, 1), ("copy", 2, 2), ("swap", 4, 2),
+                                          ("rot", 4, 2), ("dot", 2, 2), ("asum", 1, 1), ("nrm2", 1, 1), ("iamax", 1, 1)):
+                    ws = nvec * span * s
+
+                    def make_call(nbuf, r=r, nvec=nvec, span=span, n=n, inc=inc):
+                        nbuf = max(1, min(nbuf, pool.numel() // (nvec * span)))
+                        def call(k):
+                            x = pool[k * nvec * span:(k * nvec + 1) * span]
+                            y = pool[(k * nvec + 1) * span:(k * nvec + 2) * span] if nvec == 2 else None
+                            if r == "axpy":
+                                b2.axpy(ctx, n, 1e-3, x, inc, y, inc)
+                            elif r == "scal":
+                                b2.scal(ctx, n, -1.0, x, inc)
+                            elif r == "copy":
+                                b2.copy(ctx, n, x, inc, y, inc)
+                            elif r == "swap":
+                                b2.swap(ctx, n, x, inc, y, inc)
+                            elif r == "rot":
+                                b2.rot(ctx, n, x, inc, y, inc, 0.6, 0.8)
+                            elif r == "dot":
+                                b2.dot(ctx, n, x, inc, y, inc, res[0:1])
+                            elif r == "asum":
+                                b2.asum(ctx, n, x, inc, res[1:2])
+                            elif r == "nrm2":
+                                b2.nrm2(ctx, n, x, inc, res[2:3])
+                            else:
+                                b2.iamax(ctx, n, x, inc, ires)
+                        call.nbuf = nbuf
+                        return call
+                    measure(f"{r}_{dt}_n2^{lg}_inc{inc}", make_call, ws, per_elem * n * s * inc,
+                            max_sets=pool.numel() // (nvec * span))
+        del pool
+        torch.cuda.empty_cache()
+
+    # ---- gemv / ger (row-major, lda = n)
+    for dt, s in (("f32", 4), ("f64", 8)):
+        for m, n in ((4096, 4096), (16384, 16384), (1 << 20, 64), (64, 1 << 20)):
+            ws = m * n * s
+            nsets = 1 if ws >= l2 else -(-2 * l2 // ws) + 1
+            a = synth.vector_torch(0, 21, nsets * m * n, tdt[dt], device).view(nsets, m * n)
+            xv = synth.vector_torch(0, 22, max(m, n), tdt[dt], device)
+            yv = synth.vector_torch(0, 23, max(m, n), tdt[dt], device)
+            for tr, tn in ((NOTR, "n"), (TR, "t")):
+                for beta in (0.0, 0.5):
+                    mk = lambda nbuf, tr=tr, beta=beta: (lambda k: b2.gemv(ctx, ROW, tr, m, n, 1.25, a[k % nsets], n, xv, 1,
+                                                                           beta, yv, 1))
+                    ylen = m if tr == NOTR else n
+                    measure(f"gemv_{tn}_{dt}_{m}x{n}_beta{beta}", mk, ws, (m * n + m + n + (ylen if beta else 0)) * s,
+                            max_sets=nsets)
+            mk = lambda nbuf: (lambda k: b2.ger(ctx, ROW, m, n, 1e-3, xv, 1, yv, 1, a[k % nsets], n))
+            measure(f"ger_{dt}_{m}x{n}", mk, ws, (2 * m * n + m + n) * s, max_sets=nsets)
+            del a
+            torch.cuda.empty_cache()
+
+    # ---- symv / trmv / trsv
+    for dt, s in (("f32", 4), ("f64", 8)):
+        for n in (1024, 8192, 32768):
+            ws = n * n * s  # the buffer holds the full square; the routines touch one triangle of it
+            tri = n * (n + 1) // 2
+            nsets = 1 if ws // 2 >= l2 else -(-2 * l2 // (ws // 2)) + 1
+            a = synth.matrix_torch(0, 24, n, n, n, tdt[dt], device, tri_n=n).unsqueeze(0)
+            if nsets > 1:
+                a = a.repeat(nsets, 1, 1)
+            x0 = synth.vector_torch(0, 25, n, tdt[dt], device)
+            xv, yv = x0.clone(), x0.clone()
+            for ul, un in ((UP, "u"), (LO, "l")):
+                mk = lambda nbuf, ul=ul: (lambda k: b2.symv(ctx, ROW, ul, n, 1.25, a[k % nsets], n, x0, 1, 0.5, yv, 1))
+                measure(f"symv_{un}_{dt}_n{n}", mk, ws // 2, (tri + 3 * n) * s, max_sets=nsets)
+                for tr, tn in ((NOTR, "n"), (TR, "t")):
+                    for dg, dn in ((NONU, "n"), (UNIT, "u")):
+                        t = tri - (n if dg == UNIT else 0)
+                        # (both work in place: a copy launch inside the bracket restores their vector)
+                        def mk_trmv(nbuf, ul=ul, tr=tr, dg=dg):
+                            def call(k):
+                                b2.copy(ctx, n, x0, 1, xv, 1)
+                                b2.trmv(ctx, ROW, ul, tr, dg, n, a[k % nsets], n, xv, 1)
+                            return call
+                        measure(f"trmv_{un}{tn}{dn}_{dt}_n{n}", mk_trmv, ws // 2, (t + 2 * n) * s, max_sets=nsets)
+                        def mk_trsv(nbuf, ul=ul, tr=tr, dg=dg):
+                            def call(k):
+                                b2.copy(ctx, n, x0, 1, xv, 1)
+                                b2.trsv(ctx, ROW, ul, tr, dg, n, a[k % nsets], n, xv, 1)
+                            return call
+                        measure(f"trsv_{un}{tn}{dn}_{dt}_n{n}", mk_trsv, ws // 2, (t + 2 * n) * s, max_sets=nsets)
+            assert ctx.device_status() == 0, "a trsv wait timed out"
+            del a
+            torch.cuda.empty_cache()
+    return {"note": "size sweeps beside the headline set; `l2` says whether a figure is an HBM one; bytes = "
+                    "algorithmic bytes of the call (touched sectors for increment 2); trmv / trsv rows include the "
+                    "copy launch that restores their vector",
+            "l2_bytes": l2, "rows": rows}
+
+
 def e2e_leg(wl: GpuWorkload, steps: int):
     """Same metric through the C ABI with HOST data: per variant, pinned host -> device copies of
     its inputs, the call, and a device -> host read of its outputs, all inside the timed bracket."""
@@ -521,7 +696,8 @@ def aggregate(specs, med_ms, world, peak):
     for sp, t in zip(specs, med_ms):
         gbs = sp["touched"] / (t * 1e-3) / 1e9
         rows.append({"name": sp["name"], "family": sp["family"], "ms": t, "gbs": gbs,
-                     "gbs_useful": sp["useful"] / (t * 1e-3) / 1e9, "frac": gbs / peak})
+                     "gbs_useful": sp["useful"] / (t * 1e-3) / 1e9, "frac": gbs / peak,
+                     "frac_nominal": gbs / NOMINAL_PEAK_GBS})
     return rows, world * geomean([r["gbs"] for r in rows])
 
 
@@ -559,6 +735,8 @@ def main():
                                                    "strings (tuning runs; the headline run uses all)")
     ap.add_argument("--next-only", action="store_true", help="time only the rows built after the headline set "
                                                              "(--filter then selects among those)")
+    ap.add_argument("--configs", action="store_true", help="time the size sweeps beside the headline set (rows go "
+                                                           "to the table file; --filter selects among them)")
     ap.add_argument("--table", default=None, help="where the per-variant table (JSON) is written "
                                                   "(default: bench_table.json in the run's output folder)")
     args = ap.parse_args()
@@ -579,6 +757,20 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     from paper_2411_07211_b200 import binding as b2
+    if args.configs:
+        if world > 1:
+            raise SystemExit("--configs is a single-GPU run")
+        peak, peak_src = peak_gbs()
+        table = configs_leg(device, peak, max(5, min(args.steps, 10)), args.filter)
+        table["peak_gbs"], table["peak_source"] = peak, peak_src
+        path = args.table or os.path.join(ROOT, "gpurun_out", "bench_configs_table.json")
+        os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+        with open(path, "w") as f:
+            json.dump(table, f, indent=1)
+        hbm = [r["frac"] for r in table["rows"] if r["l2"].startswith("cold")]
+        print(json.dumps({"configs_rows": len(table["rows"]), "geomean_frac_cold_rows": round(geomean(hbm), 4),
+                          "table": os.path.relpath(path, ROOT)}))
+        return
     if args.next_only:
         if world > 1:
             raise SystemExit("--next-only is a single-GPU profiling aid")
@@ -657,6 +849,7 @@ def main():
                          "through L2 by a read-only kernel before every variant (clean lines only)", "bytes": "touched sectors (span bytes)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "geomean_frac_of_peak": value / world / peak,
+        "geomean_frac_of_nominal_8tbs": value / world / NOMINAL_PEAK_GBS,
         "geomean_frac_of_peak_without_trsv": geomean([r["frac"] for r in no_trsv]),
         "geomean_frac_by_family": {k: geomean([r["frac"] for r in rows if r["family"] == k]) for k in fam},
         "min_variant": min(rows, key=lambda r: r["frac"])["name"],
@@ -670,9 +863,23 @@ def main():
         scale = 16
         t0 = time.perf_counter()
         res = oracle_pass(scale)
+        t_one = time.perf_counter() - t0
         out["cpu_baseline"] = {"value": geomean([r[1] for r in res]), "unit": "GB/s", "cores": 1, "kind": "oracle",
                                "sample": f"every variant once at 1/{scale} of the bench element counts "
-                                         f"({time.perf_counter() - t0:.1f} s of CPU work)"}
+                                         f"({t_one:.1f} s of CPU work)"}
+        # second figure, context only: the same loops with an OpenMP parallel-for over the outer
+        # index on every host core (trsv and iamax stay serial)
+        try:
+            from oracle import blas_oracle as orc
+            orc.use_all_cores(True)
+            oracle_pass(scale)  # starts the thread pool, touches the pages
+            res_all = oracle_pass(scale)
+            out["cpu_baseline"]["all_cores"] = {"value": geomean([r[1] for r in res_all]), "unit": "GB/s",
+                                                "cores": os.cpu_count(), "kind": "oracle loops + OpenMP parallel-for"}
+        except Exception as e:  # no OpenMP on the box: the one-core figure stands alone
+            out["cpu_baseline"]["all_cores"] = {"unavailable": str(e)[:80]}
+        finally:
+            orc.use_all_cores(False)
     else:
         out["cpu_baseline"] = None
     table = dict(out)

@@ -23,6 +23,9 @@ UPPER, LOWER = 121, 122
 NON_UNIT, UNIT = 131, 132
 
 _lib = None
+_omp = False  # True: calls go to the OpenMP copy (the bench's all-cores baseline; timing only)
+_LIB_OMP_PATH = os.path.join(_HERE, "libblas_oracle_omp.so")
+_lib_omp = None
 
 
 def build(force: bool = False) -> str:
@@ -38,8 +41,33 @@ def build(force: bool = False) -> str:
     return _LIB_PATH
 
 
+def build_omp(force: bool = False) -> str:
+    """The same source with ORACLE_OMP defined: an OpenMP parallel-for on the outermost independent
+    loop of each routine (trsv, iamax and the float-only dots stay serial).  Timing only."""
+    stale = force or not os.path.exists(_LIB_OMP_PATH) or any(
+        os.path.getmtime(s) > os.path.getmtime(_LIB_OMP_PATH) for s in _SRC)
+    if stale:
+        tmp = _LIB_OMP_PATH + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-DORACLE_OMP", "-ffp-contract=off", "-fno-fast-math", "-Wall", "-shared", "-fPIC",
+             _SRC[0], "-o", tmp, "-lm"])
+        os.replace(tmp, _LIB_OMP_PATH)
+    return _LIB_OMP_PATH
+
+
+def use_all_cores(on: bool) -> None:
+    """Routes the calls of this module to the OpenMP copy (True) or back to the oracle proper."""
+    global _omp
+    _omp = bool(on)
+
+
 def lib():
-    global _lib
+    global _lib, _lib_omp
+    if _omp:
+        if _lib_omp is None:
+            _lib_omp = ctypes.CDLL(build_omp())
+            _lib_omp.oracle_wide_bytes.restype = ctypes.c_int
+        return _lib_omp
     if _lib is None:
         _lib = ctypes.CDLL(build())
         _lib.oracle_wide_bytes.restype = ctypes.c_int

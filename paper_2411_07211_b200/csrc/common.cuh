@@ -219,7 +219,8 @@ enum Knob {
   kKnobTrsvOwners = 13,        // blocks that own rows when helpers run (the rest of the SMs help)
   kKnobTriTile = 15,           // symv / trmv on aligned matrices: 1 = register-tile kernel, 0 = general tile kernel
   kKnobTrsvPmFrom = 14,        // first block row whose last tile is premultiplied by the inverse diagonal block
-  kKnobCount = 16
+  kKnobTriTileUnit = 16,       // tiles per unit of that kernel: 0 = by size, else 1, 2 or 4
+  kKnobCount = 24
 };
 int64_t knob(int id);
 

@@ -26,27 +26,24 @@ namespace tt {
 
 // (measured: wider, flatter tiles -- 64 x 256 or 32 x 512 floats -- are slower here, they waste
 // more of the tiles that the diagonal cuts and make the units coarser)
+constexpr int kRing = 3;       // tiles (64 KB each) in the shared-memory ring
 constexpr int kNR = 8;         // rows of a tile a thread holds
 constexpr int kNP = 2;         // packs of each row a thread holds (16 lanes side by side, kNP groups of them)
 constexpr int kTR = 16 * kNR;  // tile rows
 constexpr int kUnitMax = 4;    // tiles per unit at most (1, 2 or 4)
-constexpr int kRing = 3;      // tiles (64 KB each) in the shared-memory ring
 constexpr int kMaxMajor = 2048;  // block rows (or column tiles) the unit table can hold
 
-// Elements of the queue of x values: one slot per unit that can be in flight (kRing / unit + 2
-// units of `unit` tiles each), sized for the worst unit length.
+// Elements of the queue of x values: one slot per unit that can be in flight.  The producer runs
+// up to kRing tiles ahead of the consumer and a unit may hold a single tile (the first or last
+// unit of a row), so kRing + 1 units can be open at once; a slot is sized for the longest unit.
+constexpr int kSlots = kRing + 1;
 template <typename T, bool WALK_ROWS, bool ROWS_OF_X>
 __host__ __device__ constexpr int kSlotElems() {
   constexpr int TC = 16 * kNP * VecLen<T>::value;
   // along the walking direction a slot holds unit * tile extent values, across it one tile extent
   constexpr int ext = ROWS_OF_X ? kTR : TC;
   constexpr bool along = ROWS_OF_X != WALK_ROWS;
-  int worst = 0;
-  for (int unit = 1; unit <= kUnitMax; unit *= 2) {
-    const int need = (kRing / unit + 2) * (along ? unit : 1) * ext;
-    worst = need > worst ? need : worst;
-  }
-  return worst;
+  return kSlots * (along ? kUnitMax : 1) * ext;
 }
 
 template <typename T>
@@ -128,7 +125,7 @@ __global__ void __launch_bounds__(kThreads, 1) tri_tile_kernel(const TileArgs<T>
   const int rg = ct >> 4, cg = ct & 15;
   const int nmajor = WALK_ROWS ? p.nbr : p.nct;
   const int nunits = p.prefix[nmajor];
-  const int nslots = kRing / p.unit + 2;  // units that can be between the two cursors, plus one
+  constexpr int nslots = kSlots;
   const int xr_stride = WALK_ROWS ? kTR : p.unit * kTR, xc_stride = WALK_ROWS ? p.unit * TC : TC;
   const int64_t row_step = p.lda;                              // elements between a thread's rows
   const int64_t thread_off = (int64_t)(rg * HR) * p.lda + V * cg;  // this thread's first pack inside a half tile
@@ -426,6 +423,8 @@ static int tri_tile_run(const Launch& l, const T* a, int64_t lda, int64_t n, con
   const int64_t tiles = nbr * nct / 2;
   const int64_t want = tiles / ((int64_t)sm_count() * 16);
   args.unit = (want >= 4 && kUnitMax >= 4) ? 4 : (want >= 2 && kUnitMax >= 2) ? 2 : 1;
+  const int64_t forced = knob(kKnobTriTileUnit);
+  if (forced == 1 || forced == 2 || forced == 4) args.unit = (int)forced;
   const int nmajor = WALK_ROWS ? args.nbr : args.nct;
   int ngroups = 0;
   for (int i = 0; i < nmajor; ++i) {

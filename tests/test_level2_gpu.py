@@ -365,3 +365,33 @@ def test_trsv_moderately_conditioned(b2, ctx, dtype, c):
         assert ctx.device_status() == 0
         resid, scale = orc.trsv_residual(orc.ROW_MAJOR, uplo, trans, diag, n, a.ravel(), n, b, 1, gx.host(), 1)
         assert np.all(resid <= tol * scale), f"c={c} {uplo} {trans} {diag}: worst {np.max(resid / scale) / tol:.3f} of the bound"
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("unit", [1, 2, 4])
+def test_symv_trmv_every_unit_length(b2, ctx, dtype, unit):
+    """The tile kernel of symv / trmv cuts block rows (columns) into units of 1, 2 or 4 tiles,
+    chosen by the matrix size; here each length is forced on sizes small enough for the full oracle
+    and large enough to have rows of several units, a ragged edge, units of a single tile next to
+    full ones, and several units per block (more units than SMs)."""
+    old = b2.get_tuning(b2.KNOB_TRI_TILE_UNIT)
+    b2.set_tuning(b2.KNOB_TRI_TILE_UNIT, unit)
+    try:
+        for n in (700, 2443):
+            a = synth.matrix_np(17, 3, n, n, n, dtype, tri_n=n).ravel()
+            x, y = synth.vector_np(17, 4, n, dtype), synth.vector_np(17, 5, n, dtype)
+            ga = Guarded(a)
+            for uplo in UPLOS:
+                gx, gy = Guarded(x), Guarded(y)
+                b2.symv(ctx, orc.ROW_MAJOR, uplo, n, 1.25, ga.t, n, gx.t, 1, 0.5, gy.t, 1)
+                oy = y.copy()
+                absterms = orc.symv(orc.ROW_MAJOR, uplo, n, dtype(1.25), a, n, x, 1, dtype(0.5), oy, 1)
+                assert_close(gy.host(), oy, absterms, dtype, f"symv n={n} uplo={uplo} unit={unit}")
+                for trans, diag in itertools.product(TRANSES, DIAGS):
+                    gx = Guarded(x)
+                    b2.trmv(ctx, orc.ROW_MAJOR, uplo, trans, diag, n, ga.t, n, gx.t, 1)
+                    ox = x.copy()
+                    absterms = orc.trmv(orc.ROW_MAJOR, uplo, trans, diag, n, a, n, ox, 1)
+                    assert_close(gx.host(), ox, absterms, dtype, f"trmv n={n} {uplo} {trans} {diag} unit={unit}")
+    finally:
+        b2.set_tuning(b2.KNOB_TRI_TILE_UNIT, old)
