@@ -735,6 +735,8 @@ def main():
                                                    "strings (tuning runs; the headline run uses all)")
     ap.add_argument("--next-only", action="store_true", help="time only the rows built after the headline set "
                                                              "(--filter then selects among those)")
+    ap.add_argument("--knob", action="append", default=[], metavar="ID=VALUE",
+                    help="set a tuning knob of the library before timing (tuning runs; the headline run sets none)")
     ap.add_argument("--configs", action="store_true", help="time the size sweeps beside the headline set (rows go "
                                                            "to the table file; --filter selects among them)")
     ap.add_argument("--table", default=None, help="where the per-variant table (JSON) is written "
@@ -757,6 +759,9 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     from paper_2411_07211_b200 import binding as b2
+    for kv in args.knob:
+        kid, val = kv.split("=")
+        b2.set_tuning(int(kid), int(val))
     if args.configs:
         if world > 1:
             raise SystemExit("--configs is a single-GPU run")

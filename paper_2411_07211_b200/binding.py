@@ -29,8 +29,7 @@ KNOB_L1_BLOCKS_PER_SM, KNOB_GEMV_N_TILE_BYTES, KNOB_GEMV_T_ROWS, KNOB_TRI_ROWS =
 KNOB_GER_ROWS, KNOB_USE_PDL, KNOB_TRSV_DEBUG_SKIP, KNOB_TRI_WIDE = 4, 5, 6, 7
 KNOB_TRSV_PREFETCH_BYTES = 8
 KNOB_TRSV_FRONT, KNOB_TRSV_CLUSTER = 9, 10
-KNOB_TRSV_HELP_NEAR, KNOB_TRSV_HELP_CHUNK, KNOB_TRSV_OWNERS = 11, 12, 13
-KNOB_TRSV_PM_FROM, KNOB_TRI_TILE, KNOB_TRI_TILE_UNIT = 14, 15, 16
+KNOB_TRSV_PM_FROM, KNOB_TRI_TILE, KNOB_TRI_TILE_UNIT = 11, 12, 13
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libb2blas.so")
 

@@ -15,11 +15,9 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobTrsvPrefetchBytes */ 48 << 20,
     /* kKnobTrsvFront       */ 2,
     /* kKnobTrsvCluster     */ 0,
-    /* kKnobTrsvHelpNear    */ 12,
-    /* kKnobTrsvHelpChunk   */ 8,
-    /* kKnobTrsvOwners      */ 48,
-    /* kKnobTrsvPmFrom      */ 10,
+    /* kKnobTrsvPmFrom      */ 16,
     /* kKnobTriTile         */ 1,
+    /* kKnobTriTileUnit     */ 0,
 };
 
 unsigned long long g_launch_count = 0;

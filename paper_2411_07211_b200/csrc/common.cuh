@@ -20,14 +20,12 @@ constexpr int kWarps = kThreads / 32;
 //   word 0      : ticket counter of the level-1 reductions
 //   word 16     : ticket counter of trsv (next block-row to hand out)
 //   word 17     : trsv "blocks finished" counter
-//   word 18     : sub-block trsv: ticket counter of the helper units
 //   word 19     : sub-block trsv: abort flag (stays up after a timeout until the workspace is reset)
 // Scratch (partials, trsv flags) starts at kCtlBytes.
 constexpr size_t kCtlBytes = 4096;
 constexpr int kCtlReduceTicket = 0;
 constexpr int kCtlTrsvTicket = 16;
 constexpr int kCtlTrsvDone = 17;
-constexpr int kCtlTrsvHelpTicket = 18;
 constexpr int kCtlTrsvAbort = 19;  // sub-block trsv: raised when a bounded wait ran out
 
 // ---------------------------------------------------------------------------------------
@@ -214,13 +212,10 @@ enum Knob {
   kKnobTrsvPrefetchBytes = 8,  // total L2 bytes trsv blocks may prefetch ahead of the front
   kKnobTrsvFront = 9,          // 0: block-row trsv kernel only; 1: sub-block kernel for row-type views; 2: for all views
   kKnobTrsvCluster = 10,       // sub-block trsv in clusters of 8 block rows: 0 never, 1 float only, 2 always
-  kKnobTrsvHelpNear = 11,      // tiles next to the diagonal an owner block keeps at least (0: no helper blocks)
-  kKnobTrsvHelpChunk = 12,     // tiles per helper unit (even)
-  kKnobTrsvOwners = 13,        // blocks that own rows when helpers run (the rest of the SMs help)
-  kKnobTriTile = 15,           // symv / trmv on aligned matrices: 1 = register-tile kernel, 0 = general tile kernel
-  kKnobTrsvPmFrom = 14,        // first block row whose last tile is premultiplied by the inverse diagonal block
-  kKnobTriTileUnit = 16,       // tiles per unit of that kernel: 0 = by size, else 1, 2 or 4
-  kKnobCount = 24
+  kKnobTrsvPmFrom = 11,        // first block row whose last tile is premultiplied by the inverse diagonal block
+  kKnobTriTile = 12,           // tile kernel with the shared-memory ring: 0 never, 1 symv and the trmv cases it wins, 2 symv and every trmv
+  kKnobTriTileUnit = 13,       // tiles per unit of that kernel: 0 = by size, else 1, 2 or 4
+  kKnobCount = 16
 };
 int64_t knob(int id);
 

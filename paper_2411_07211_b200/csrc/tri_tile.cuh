@@ -46,7 +46,9 @@ __host__ __device__ constexpr int kSlotElems() {
   return kSlots * (along ? kUnitMax : 1) * ext;
 }
 
-template <typename T>
+// CAP: entries of the unit table.  The table travels in the kernel parameters; matrices of up to
+// 128 block rows (columns) use the short form, whose parameter block is a tenth of the long one.
+template <typename T, int CAP>
 struct TileArgs {
   const T* a;
   int64_t lda, n;
@@ -60,7 +62,7 @@ struct TileArgs {
   T alpha, beta;
   T* y;
   int64_t incy;
-  int prefix[kMaxMajor + 1];  // units before block row (column tile) i; the last entry is their total
+  int prefix[CAP + 1];  // units before block row (column tile) i; the last entry is their total
 };
 
 // First and last column tile of block row I that meets the triangle.
@@ -107,8 +109,8 @@ __device__ __forceinline__ void cp_async_wait() {
 // next kRing - 1 tiles (also those of the block's next units) are in flight while a tile is
 // multiplied.  Edge tiles use the same copies with a byte count that zero-fills what lies outside
 // the matrix.  The x values of a unit travel the same way.
-template <typename T, bool ROW, bool COL, int TRI, bool UNIT, bool SYM>
-__global__ void __launch_bounds__(kThreads, 1) tri_tile_kernel(const TileArgs<T> p) {
+template <typename T, int CAP, bool ROW, bool COL, int TRI, bool UNIT, bool SYM>
+__global__ void __launch_bounds__(kThreads, 1) tri_tile_kernel(const TileArgs<T, CAP> p) {
   constexpr int V = VecLen<T>::value, TC = 16 * kNP * V, NR = kNR, HR = NR / 2, NP = kNP, TP = NR * NP;
   constexpr bool WALK_ROWS = ROW;  // column-sum-only kinds walk down a block column
   constexpr int XCU = WALK_ROWS ? kUnitMax * TC : TC;  // most column values a unit needs
@@ -338,13 +340,18 @@ __global__ void __launch_bounds__(kThreads, 1) tri_tile_kernel(const TileArgs<T>
 }
 
 // y_i = alpha * (row partials of i + column partials of i) + beta * y_i, the partials added in a
-// fixed order.  A block of 32 warps serves 32 consecutive outputs (one per lane, so every load is
+// fixed order.  A block of 32 (16) warps serves 32 consecutive outputs (one per lane, so every load is
 // a coalesced row segment of a partial array); warp w takes partials w, w + 32, ... -- a handful
 // of independent loads, all in flight at once -- and warp 0 adds the 32 sums in warp order.
-constexpr int kFinWarps = 32;
-template <typename T, bool ROW, bool COL, int TRI>
-__global__ void __launch_bounds__(kFinWarps * 32) tri_tile_finalize(const TileArgs<T> p) {
-  constexpr int V = VecLen<T>::value, TC = 16 * kNP * V;
+// (16 warps in double precision: the block's shared memory must fit beside a tile-kernel block
+// that is still running, or the early launch waits for it to leave)
+template <typename T>
+__host__ __device__ constexpr int fin_warps() {
+  return sizeof(T) == 8 ? 16 : 32;
+}
+template <typename T, int CAP, bool ROW, bool COL, int TRI>
+__global__ void __launch_bounds__(fin_warps<T>() * 32) tri_tile_finalize(const TileArgs<T, CAP> p) {
+  constexpr int V = VecLen<T>::value, TC = 16 * kNP * V, kFinWarps = fin_warps<T>();
   constexpr bool WALK_ROWS = ROW;
   __shared__ T part[kFinWarps][33];
   grid_dep_wait();
@@ -402,16 +409,13 @@ constexpr size_t tile_smem_bytes() {
 // Launches both kernels.  *handled is false (nothing launched) when the matrix is not 16-byte
 // aligned, too large for the unit table, or the partials do not fit the workspace: the caller
 // then uses the general tile kernel.
-template <typename T, bool ROW, bool COL, int TRI, bool UNIT, bool SYM>
-static int tri_tile_run(const Launch& l, const T* a, int64_t lda, int64_t n, const T* x, int64_t incx, T alpha, T beta,
-                        T* y, int64_t incy, bool* handled) {
+template <typename T, int CAP, bool ROW, bool COL, int TRI, bool UNIT, bool SYM>
+static int tri_tile_run_cap(const Launch& l, const T* a, int64_t lda, int64_t n, const T* x, int64_t incx, T alpha, T beta,
+                            T* y, int64_t incy, bool* handled) {
   constexpr int V = VecLen<T>::value, TC = 16 * kNP * V;
   constexpr bool WALK_ROWS = ROW;
-  *handled = false;
-  if (!aligned_to(a, 16) || lda % V != 0) return B2_STATUS_OK;
   const int64_t nbr = (n + kTR - 1) / kTR, nct = (n + TC - 1) / TC;
-  if ((WALK_ROWS ? nbr : nct) > kMaxMajor) return B2_STATUS_OK;
-  TileArgs<T> args = {};
+  TileArgs<T, CAP> args = {};
   args.a = a;
   args.lda = lda;
   args.n = n;
@@ -446,7 +450,7 @@ static int tri_tile_run(const Launch& l, const T* a, int64_t lda, int64_t n, con
   args.y = y;
   args.incy = incy;
   constexpr size_t smem = tile_smem_bytes<T, ROW, COL>();
-  auto kern = tri_tile_kernel<T, ROW, COL, TRI, UNIT, SYM>;
+  auto kern = tri_tile_kernel<T, CAP, ROW, COL, TRI, UNIT, SYM>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     (void)cudaGetLastError();
     return B2_STATUS_OK;
@@ -458,15 +462,27 @@ static int tri_tile_run(const Launch& l, const T* a, int64_t lda, int64_t n, con
   if (int st = check_launch()) return st;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)((n + 31) / 32));
-  cfg.blockDim = dim3(kFinWarps * 32);
+  cfg.blockDim = dim3(fin_warps<T>() * 32);
   cfg.stream = l.stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = knob(kKnobUsePdl) ? 1 : 0;
-  cudaLaunchKernelEx(&cfg, tri_tile_finalize<T, ROW, COL, TRI>, args);
+  cudaLaunchKernelEx(&cfg, tri_tile_finalize<T, CAP, ROW, COL, TRI>, args);
   return check_launch();
+}
+
+template <typename T, bool ROW, bool COL, int TRI, bool UNIT, bool SYM>
+static int tri_tile_run(const Launch& l, const T* a, int64_t lda, int64_t n, const T* x, int64_t incx, T alpha, T beta,
+                        T* y, int64_t incy, bool* handled) {
+  constexpr int V = VecLen<T>::value, TC = 16 * kNP * V;
+  *handled = false;
+  if (!aligned_to(a, 16) || lda % V != 0) return B2_STATUS_OK;
+  const int64_t nmajor = ROW ? (n + kTR - 1) / kTR : (n + TC - 1) / TC;
+  if (nmajor > kMaxMajor) return B2_STATUS_OK;
+  if (nmajor <= 128) return tri_tile_run_cap<T, 128, ROW, COL, TRI, UNIT, SYM>(l, a, lda, n, x, incx, alpha, beta, y, incy, handled);
+  return tri_tile_run_cap<T, kMaxMajor, ROW, COL, TRI, UNIT, SYM>(l, a, lda, n, x, incx, alpha, beta, y, incy, handled);
 }
 
 }  // namespace tt

@@ -20,13 +20,6 @@
 //      instruction fetches on the critical path; everything between "x_{k-1} is visible" and
 //      "x_k is published" is therefore code the block has been executing on every tile,
 //      including the publishing stores (predicated off on the earlier trips).
-// Long block rows are shared.  Streaming row k alone takes one SM k tiles, and the late rows would
-// finish long after the front could have reached them; so an owner keeps only the last tiles of
-// its row (those whose x arrives while it runs) and HELPER blocks take the rest in units of
-// `chunk` tiles (row k, columns c*chunk .. c*chunk+chunk-1).  Units are drawn in column order --
-// a unit is runnable as soon as the front has passed its columns, the rows closest to the front
-// first -- and a unit adds the partial of the unit before it in the same row, so the owner
-// reads ONE vector of row sums, formed in a fixed order (results stay bit-reproducible).
 // Values cross SMs as 64-bit words {32 payload bits, 32-bit call tag}: data and ready flag
 // are one store, and the consumer polls the data itself.  Every wait is bounded: when a
 // budget runs out the thread records B2_STATUS_TIMEOUT, raises an abort word in the control
@@ -66,12 +59,6 @@ struct FrontArgs {
   int* device_status;
   int debug_skip;
   int pm_from;  // first row (solve order) that premultiplies its last tile
-  // helper units (all zero: no helpers, every block owns rows)
-  int near_min;       // an owner keeps the last near_min .. near_min + chunk - 1 tiles of its row
-  int chunk;          // tiles per helper unit
-  int owner_groups;   // blocks (clusters) with index below this own rows, the others are helpers
-  unsigned n_units;
-  unsigned long long* hp;  // unit partials: [unit][NB] values as tagged words
 };
 
 
@@ -157,31 +144,6 @@ __device__ __forceinline__ double decode(const unsigned long long* w, double) {
   return __longlong_as_double((long long)(((unsigned long long)(unsigned)w[1] << 32) | (unsigned)w[0]));
 }
 
-// Helper units in column order.  Column c holds the rows k >= (c + 1) * chunk + near_min, n0 of
-// them in column 0 and `chunk` fewer in each later column.
-struct Units {
-  long long n0;
-  int chunk, near_min;
-  __host__ __device__ long long before(long long c) const { return c * n0 - (long long)chunk * (c * (c - 1) / 2); }
-  __host__ __device__ long long columns() const { return n0 > 0 ? (n0 + chunk - 1) / chunk : 0; }
-  __host__ __device__ long long total() const { return before(columns()); }
-  __host__ __device__ long long id(int k, int c) const { return before(c) + k - (long long)(c + 1) * chunk - near_min; }
-  // first column tile an owner keeps (= tiles its helpers take)
-  __host__ __device__ int first_near(int k) const {
-    return (near_min > 0 && k - near_min >= chunk) ? ((k - near_min) / chunk) * chunk : 0;
-  }
-  __device__ void locate(long long u, int* k, int* c) const {
-    long long lo = 0, hi = columns() - 1;  // largest column with before(column) <= u
-    while (lo < hi) {
-      const long long mid = (lo + hi + 1) >> 1;
-      if (before(mid) <= u) lo = mid;
-      else hi = mid - 1;
-    }
-    *c = (int)lo;
-    *k = (int)(u - before(lo) + (lo + 1) * chunk + near_min);
-  }
-};
-
 // Per-thread state of the bounded waits.
 struct Waiter {
   unsigned long long budget;
@@ -215,28 +177,6 @@ struct Waiter {
       if (sleep_ns) __nanosleep(sleep_ns);
       ld_word2(ptr, w[0], w[1]);
       ld_word2(ptr + 2, w[2], w[3]);
-    }
-  }
-  // The N (1 or 2) tagged words of one value at ptr (16-byte aligned when N = 2).
-  template <int N>
-  __device__ __forceinline__ void fetch(unsigned long long (&w)[N], const unsigned long long* ptr, unsigned tag,
-                                        unsigned sleep_ns) {
-    for (;;) {
-      if (N == 1) asm volatile("ld.relaxed.gpu.u64 %0, [%1];" : "=l"(w[0]) : "l"(ptr) : "memory");
-      else ld_word2(ptr, w[0], w[N - 1]);
-      bool ok = true;
-#pragma unroll
-      for (int i = 0; i < N; ++i) ok = ok && (unsigned)(w[i] >> 32) == tag;
-      if (ok || dead) return;
-      if (--budget == 0) {
-        fail();
-        return;
-      }
-      if ((budget & 15) == 0 && ld_flag(abort_word) != 0u) {
-        dead = true;
-        return;
-      }
-      if (sleep_ns) __nanosleep(sleep_ns);
     }
   }
 };
@@ -284,14 +224,14 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
   constexpr int SP = NB + 16 / (int)sizeof(T);  // row pitch of S (rows start 16-byte aligned)
   constexpr bool CANON_LOWER = (COLTYPE == BACKWARD);  // stored triangle in the row-major view
   using P = Pack<T, V>;
-  constexpr bool PM = true;  // premultiply the last tile (see below)
+  constexpr bool PM = CS == 1;  // premultiply the last tile (see below)
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* S = reinterpret_cast<T*>(smem_raw);       // diagonal block, then its inverse (symmetric storage)
   T* Tm = S + NB * SP;                          // products in flight during the inversion
   T* Wt = S;                                    // ... and finally the inverse in the tile loader's layout
   T* Ms = Tm + (NB / 2) * (NB / 2 + 4);         // inv(D_k) * A_{k,k-1} in the same layout (the tile of the last trip)
-  T* xs = Ms + NB * SP;                         // [2][NB] x values of the current / next tile
+  T* xs = Ms + (PM ? NB * SP : 0);              // [2][NB] x values of the current / next tile
   T* rbuf = xs + 2 * NB;                        // r = b - sum, the vector of the final trip
   T* bvec = rbuf + NB;
   T* red = bvec + NB;                           // [kT / 32][NB] per-warp partial row sums (column-type views)
@@ -325,51 +265,31 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     cluster_sync_all();
   }
 
-  const Units units = {(long long)p.nb - p.chunk - p.near_min, p.chunk > 0 ? p.chunk : 1, p.near_min};
-  const bool helper_role = (int)(blockIdx.x / CS) >= p.owner_groups;
-
   for (;;) {
-    unsigned long long kk;
-    int hcol = 0;  // helper: column of the unit
-    long long unit = 0;
-    if (helper_role) {
-      // one ticket per block = one unit, in column order
-      if (ct == 0) {
-        unsigned u = 0xffffffffu;
-        if (!wt.dead && ld_flag(wt.abort_word) == 0u) u = atomicAdd(p.ctl + kCtlTrsvHelpTicket, 1u);
-        s_ticket[parity] = u;
+    // one ticket per cluster = CS consecutive block rows in solve order
+    if (rank == 0u && ct == 0) {
+      unsigned kk = 0xffffffffu;
+      if (!wt.dead && ld_flag(wt.abort_word) == 0u) kk = atomicAdd(p.ctl + kCtlTrsvTicket, 1u);
+      // abort word up (raised in this call, or left by an earlier timed-out call on a workspace
+      // that was not reset): nothing more is solved, and the caller must be able to see that
+      else if (p.device_status) atomicExch(p.device_status, (int)B2_STATUS_TIMEOUT);
+      // abort word up (raised in this call, or left by an earlier timed-out call on a workspace
+      // that was not reset): nothing more is solved, and the caller must be able to see that
+      else if (p.device_status) atomicExch(p.device_status, (int)B2_STATUS_TIMEOUT);
+      if (CS > 1) {
+        for (unsigned r = 0; r < (unsigned)CS; ++r) st_remote_u32(map_remote(&s_ticket[parity], r), kk);
+      } else {
+        s_ticket[parity] = kk;
       }
-      bar_sync(kBar, kT);
-      unit = s_ticket[parity];
-      parity ^= 1;
-      if (unit >= (long long)p.n_units) break;
-      int hk;
-      units.locate(unit, &hk, &hcol);
-      kk = (unsigned long long)hk;
-    } else {
-      // one ticket per cluster = CS consecutive block rows in solve order
-      if (rank == 0u && ct == 0) {
-        unsigned t = 0xffffffffu;
-        if (!wt.dead && ld_flag(wt.abort_word) == 0u) t = atomicAdd(p.ctl + kCtlTrsvTicket, 1u);
-        // abort word up (raised in this call, or left by an earlier timed-out call on a workspace
-        // that was not reset): nothing more is solved, and the caller must be able to see that
-        else if (p.device_status) atomicExch(p.device_status, (int)B2_STATUS_TIMEOUT);
-        if (CS > 1) {
-          for (unsigned r = 0; r < (unsigned)CS; ++r) st_remote_u32(map_remote(&s_ticket[parity], r), t);
-        } else {
-          s_ticket[parity] = t;
-        }
-      }
-      if (CS > 1) cluster_sync_all();
-      else bar_sync(kBar, kT);
-      kk = (unsigned long long)s_ticket[parity] * CS + rank;
-      parity ^= 1;
-      if (kk - rank >= (unsigned long long)p.nb) break;  // the whole cluster leaves together
-      if (kk >= (unsigned long long)p.nb) continue;     // this group has fewer than CS rows
     }
+    if (CS > 1) cluster_sync_all();
+    else bar_sync(kBar, kT);
+    const unsigned long long kk = (unsigned long long)s_ticket[parity] * CS + rank;
+    parity ^= 1;
+    if (kk - rank >= (unsigned long long)p.nb) break;  // the whole cluster leaves together
+    if (kk >= (unsigned long long)p.nb) continue;     // this group has fewer than CS rows
     const int k = (int)kk;  // position in the solve order = number of source tiles
-    const int g0 = helper_role ? 0x7fffffff : k - (int)rank;  // first row of this cluster's group
-    const int fk = units.first_near(k);  // an owner's first tile; the tiles before it are its helpers'
+    const int g0 = k - (int)rank;  // first row of this cluster's group
     const int I = BACKWARD ? p.nb - 1 - k : k;
     const int64_t r0 = (int64_t)I * NB;
     const int nbI = (int)min((int64_t)NB, p.n - r0);
@@ -459,110 +379,6 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       }
     };
 
-    // warp 0 fetches the x values a trip needs: 4 tagged words per lane, first attempt one trip ahead
-    unsigned long long xw[4] = {0, 0, 0, 0};
-    unsigned xneed = 0, xtag = p.tag;
-    const unsigned long long* xptr = p.xbuf;
-    auto x_issue = [&](int s) {
-      const int64_t xi = (int64_t)blk(s) * NB + V * lane;
-      xneed = 0;
-#pragma unroll
-      for (int e = 0; e < V; ++e)
-        if (xi + e < p.n) xneed |= ((1u << WPE) - 1u) << (e * WPE);
-      const bool local = CS > 1 && s >= g0;  // a row of this cluster: its block writes into xrecv
-      xptr = local ? xrecv + ((s - g0) * NB + V * lane) * WPE : p.xbuf + xi * WPE;
-      xtag = local ? (unsigned)s + 1u : p.tag;
-      if (xneed) {
-        ld_word2(xptr, xw[0], xw[1]);
-        ld_word2(xptr + 2, xw[2], xw[3]);
-      }
-    };
-    // warp 0: waits for the words x_issue asked for and leaves the values in dst
-    auto x_take = [&](T* dst, unsigned sleep_ns) {
-      wt.finish(xw, xptr, xneed, xtag, sleep_ns);
-      P xv;
-#pragma unroll
-      for (int e = 0; e < V; ++e) xv.v[e] = ((xneed >> (e * WPE)) & 1u) ? decode(xw + e * WPE, T(0)) : T(0);
-      *reinterpret_cast<P*>(dst + V * lane) = xv;
-    };
-    // tile (in registers) times vector (in shared memory): the sum of row `ti` of the product on the
-    // threads that own a row.  Column-type views pass one block-wide barrier inside.
-    auto tile_times = [&](const T (&cur)[E], const T* vec) -> T {
-      T s;
-      if constexpr (!COLTYPE) {
-        T xv[RS], part[RS];
-#pragma unroll
-        for (int hb = 0; hb < RS / V; ++hb) {
-          const P pk = *reinterpret_cast<const P*>(vec + hb * H + V * cg);
-#pragma unroll
-          for (int e = 0; e < V; ++e) xv[hb * V + e] = pk.v[e];
-        }
-#pragma unroll
-        for (int a = 0; a < RS; ++a) {
-          part[a] = T(0);
-#pragma unroll
-          for (int bcol = 0; bcol < RS; ++bcol) part[a] = cur[a * RS + bcol] * xv[bcol] + part[a];
-        }
-        s = multi_group_sum<16, RS>(part, lane);
-      } else {
-        P part;
-#pragma unroll
-        for (int e = 0; e < V; ++e) part.v[e] = T(0);
-#pragma unroll
-        for (int q = 0; q < JT / V; ++q) {
-          const P pk = *reinterpret_cast<const P*>(vec + warp * JT + q * V);  // the warp's columns: a broadcast
-#pragma unroll
-          for (int u = 0; u < V; ++u)
-#pragma unroll
-            for (int e = 0; e < V; ++e) part.v[e] = cur[(q * V + u) * V + e] * pk.v[u] + part.v[e];
-        }
-        *reinterpret_cast<P*>(red + warp * NB + V * lane) = part;
-        bar_sync(kBar, kT);  // (the next trip writes red only after its own first barrier)
-        s = T(0);
-        if (ct < NB) {
-#pragma unroll
-          for (int w = 0; w < kT / 32; ++w) s += red[w * NB + ct];
-        }
-      }
-      return s;
-    };
-    // two register sets take turns: while one is multiplied, the other receives the next tile
-    T tile_a[E], tile_b[E];
-
-    if (helper_role) {
-      // --- helper unit: `chunk` tiles of row k, the running sum of the row's units goes to hp[unit]
-      const int s0 = hcol * p.chunk, ns = p.chunk;
-      load_tile(tile_a, s0, true);
-      for (int j = 1; j <= p.pf_dist && j < ns; ++j) prefetch_tile(s0 + j);
-      if (warp == 0) x_issue(s0);
-      T hacc = T(0);
-      auto htrip = [&](T (&cur)[E], T (&nxt)[E], int j) {
-        T* xbuf_s = xs + (j & 1) * NB;
-        if (j + 1 < ns) load_tile(nxt, s0 + j + 1, true);
-        if (j + 1 + p.pf_dist < ns) prefetch_tile(s0 + j + 1 + p.pf_dist);
-        if (warp == 0) x_take(xbuf_s, 100u);
-        bar_sync(kBar, kT);
-        hacc += tile_times(cur, xbuf_s);
-        if (warp == 0 && j + 1 < ns) x_issue(s0 + j + 1);
-      };
-#pragma unroll 1
-      for (int j = 0; j < ns; j += 2) {
-        htrip(tile_a, tile_b, j);
-        if (j + 1 < ns) htrip(tile_b, tile_a, j + 1);
-      }
-      if (owner) {
-        T prev = T(0);
-        if (hcol > 0) {  // the unit before this one in the row was drawn earlier: a bounded wait
-          unsigned long long hw[WPE];
-          wt.template fetch<WPE>(hw, p.hp + ((size_t)units.id(k, hcol - 1) * NB + ti) * WPE, p.tag, 200u);
-          prev = decode(hw, T(0));
-        }
-        publish_if(!wt.dead, p.hp + ((size_t)unit * NB + ti) * WPE, prev + hacc, p.tag);
-      }
-      bar_sync(kBar, kT);  // xs and red are reused by the next unit
-      continue;
-    }
-
     // --- diagonal block -> S, solve order, symmetric storage (S[t][t'] = S[t'][t]); b -> bvec
     if (nbI < NB)
       for (int idx = ct; idx < NB * SP; idx += kT) S[idx] = T(0);
@@ -607,7 +423,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     for (int s = ct; s < NB; s += kT)
       if (s >= nbI) S[s * SP + s] = T(1);
     prefetch_tile(k - 1);
-    for (int s = 0; s < p.pf_dist; ++s) prefetch_tile(fk + s);
+    for (int s = 0; s < p.pf_dist; ++s) prefetch_tile(s);
     bar_sync(kBar, kT);
 
     // --- in-place inverse.  4x4 diagonal blocks by substitution (one column per thread) ...
@@ -809,14 +625,30 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     // --- along the block row.  Trips 0 .. k-2 multiply the tiles A_ks by x_s and add up; trip
     // yt = k-1 multiplies inv(D_k) by r = b - sum (y); trip k multiplies Ms by x_{k-1}: x_k = y - that.
     // (Row 0 has the single trip yt = 0 and x_0 = y.)
-    load_tile(tile_a, fk, false);
-    T bi = bvec[ti];
+    // two register sets take turns: while one is multiplied, the other receives the next tile
+    T tile_a[E], tile_b[E];
+    load_tile(tile_a, 0, false);
+    const T bi = bvec[ti];
     T racc = T(0), yreg = T(0);
-    // the trip in which the row sums of the helpers' tiles are taken over (their last unit was
-    // runnable four rows of the front earlier)
-    const int hwt = fk > 0 ? min(fk + 4, yt - 1) : -1;
-    const unsigned long long* hptr = p.hp + (fk > 0 ? ((size_t)units.id(k, fk / units.chunk - 1) * NB + ti) * WPE : 0);
-    if (warp == 0 && k > 0) x_issue(yt > fk ? fk : k - 1);  // (yt == 0 < k only with PM: the M trip's x)
+    // warp 0 fetches the x values a trip needs: 4 tagged words per lane, first attempt one trip ahead
+    unsigned long long xw[4] = {0, 0, 0, 0};
+    unsigned xneed = 0, xtag = p.tag;
+    const unsigned long long* xptr = p.xbuf;
+    auto x_issue = [&](int s) {
+      const int64_t xi = (int64_t)blk(s) * NB + V * lane;
+      xneed = 0;
+#pragma unroll
+      for (int e = 0; e < V; ++e)
+        if (xi + e < p.n) xneed |= ((1u << WPE) - 1u) << (e * WPE);
+      const bool local = CS > 1 && s >= g0;  // a row of this cluster: its block writes into xrecv
+      xptr = local ? xrecv + ((s - g0) * NB + V * lane) * WPE : p.xbuf + xi * WPE;
+      xtag = local ? (unsigned)s + 1u : p.tag;
+      if (xneed) {
+        ld_word2(xptr, xw[0], xw[1]);
+        ld_word2(xptr + 2, xw[2], xw[3]);
+      }
+    };
+    if (warp == 0 && k > 0) x_issue(yt > 0 ? 0 : k - 1);  // (yt == 0 < k only with PM: the M trip's x)
 
     auto trip = [&](T (&cur)[E], T (&nxt)[E], int it) {
       const bool is_y = it == yt;
@@ -830,18 +662,53 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
       prefetch_tile(it + 1 + p.pf_dist);
       if (warp == 0 && !is_y) {
         const int dist = k - srow;  // rows between this block and the producer of the x
-        x_take(xbuf_s, dist > 2 ? (unsigned)min((dist - 2) * 200, 2000) : 0u);
+        wt.finish(xw, xptr, xneed, xtag, dist > 2 ? (unsigned)min((dist - 2) * 200, 2000) : 0u);
+        P xv;
+#pragma unroll
+        for (int e = 0; e < V; ++e) xv.v[e] = ((xneed >> (e * WPE)) & 1u) ? decode(xw + e * WPE, T(0)) : T(0);
+        *reinterpret_cast<P*>(xbuf_s + V * lane) = xv;
       }
       bar_sync(kBar, kT);
-      const T s = tile_times(cur, is_y ? rbuf : xbuf_s);
+      const T* vec = is_y ? rbuf : xbuf_s;
+      T s;
+      if constexpr (!COLTYPE) {
+        T xv[RS], part[RS];
+#pragma unroll
+        for (int hb = 0; hb < RS / V; ++hb) {
+          const P pk = *reinterpret_cast<const P*>(vec + hb * H + V * cg);
+#pragma unroll
+          for (int e = 0; e < V; ++e) xv[hb * V + e] = pk.v[e];
+        }
+#pragma unroll
+        for (int a = 0; a < RS; ++a) {
+          part[a] = T(0);
+#pragma unroll
+          for (int bcol = 0; bcol < RS; ++bcol) part[a] = cur[a * RS + bcol] * xv[bcol] + part[a];
+        }
+        s = multi_group_sum<16, RS>(part, lane);
+      } else {
+        P part;
+#pragma unroll
+        for (int e = 0; e < V; ++e) part.v[e] = T(0);
+#pragma unroll
+        for (int q = 0; q < JT / V; ++q) {
+          const P pk = *reinterpret_cast<const P*>(vec + warp * JT + q * V);  // the warp's columns: a broadcast
+#pragma unroll
+          for (int u = 0; u < V; ++u)
+#pragma unroll
+            for (int e = 0; e < V; ++e) part.v[e] = cur[(q * V + u) * V + e] * pk.v[u] + part.v[e];
+        }
+        *reinterpret_cast<P*>(red + warp * NB + V * lane) = part;
+        bar_sync(kBar, kT);  // (the next trip writes red only after its own first barrier)
+        s = T(0);
+        if (ct < NB) {
+#pragma unroll
+          for (int w = 0; w < kT / 32; ++w) s += red[w * NB + ct];
+        }
+      }
       const T out = is_m ? yreg - s : s;
       if (is_y) yreg = s;
       if (it < yt) racc += s;
-      if (it == hwt && owner) {  // the helpers' share of the row sums (a bounded wait, normally long over)
-        unsigned long long hw[WPE];
-        wt.template fetch<WPE>(hw, hptr, p.tag, 0u);
-        bi -= decode(hw, T(0));
-      }
       if (owner && it < yt) rbuf[ti] = bi - racc;
       {  // publishing stores: fetched on every trip, performed on the last
         const bool real = crit && owner && row_ok && !wt.dead && k != p.debug_skip;
@@ -866,7 +733,7 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     int ntrips = k + 1;
     asm volatile("" : "+r"(ntrips));  // loops of two trips, not peeled copies of the last ones
 #pragma unroll 1
-    for (int it = fk; it < ntrips; it += 2) {  // (fk is even: a whole number of helper units)
+    for (int it = 0; it < ntrips; it += 2) {
       trip(tile_a, tile_b, it);
       if (it + 1 < ntrips) trip(tile_b, tile_a, it + 1);
     }
@@ -879,7 +746,6 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     const unsigned d = atomicAdd(p.ctl + kCtlTrsvDone, 1u);
     if (d == gridDim.x - 1) {
       p.ctl[kCtlTrsvTicket] = 0u;
-      p.ctl[kCtlTrsvHelpTicket] = 0u;
       p.ctl[kCtlTrsvDone] = 0u;
     }
   }
@@ -889,32 +755,16 @@ template <typename T>
 constexpr size_t front_smem_bytes(int cs) {
   constexpr int NB = Geo<T>::NB;
   constexpr int SP = NB + 16 / (int)sizeof(T);
-  return sizeof(T) * (size_t)(2 * NB * SP + (NB / 2) * (NB / 2 + 4) + (4 + kT / 32) * NB) +
+  return sizeof(T) * (size_t)((cs > 1 ? 1 : 2) * NB * SP + (NB / 2) * (NB / 2 + 4) + (4 + kT / 32) * NB) +
          (cs > 1 ? (size_t)cs * NB * Words<T>::N * 8 : 0);
 }
 
 constexpr int kCluster = 8;
 
-// Fills in the helper fields of the arguments for a grid of `groups` blocks (or clusters): with
-// helper units, at most kKnobTrsvOwners blocks own rows and the rest of the grid helps.
-template <typename T>
-static void split_roles(FrontArgs<T>& args, int groups, int owner_cap, bool helpers) {
-  if (owner_cap < 1) owner_cap = 1;
-  if (helpers && groups > owner_cap) {
-    args.owner_groups = owner_cap;
-  } else {
-    args.owner_groups = groups;
-    args.near_min = 0;
-    args.n_units = 0;
-  }
-}
-
 // Launches the kernel; with clusters when the device can hold at least one (the grid is then a
 // whole number of clusters, no more than can be resident), else block by block.
 template <typename T, bool COLTYPE, bool BACKWARD, bool UNIT>
-static int launch_one(const Launch& l, FrontArgs<T> args, int nb, bool want_cluster) {
-  const bool helpers = args.n_units > 0;
-  const int owners = (int)knob(kKnobTrsvOwners);
+static int launch_one(const Launch& l, const FrontArgs<T>& args, int nb, bool want_cluster) {
   if (want_cluster) {
     constexpr size_t smem = front_smem_bytes<T>(kCluster);
     auto kern = trsv_front_kernel<T, COLTYPE, BACKWARD, UNIT, kCluster>;
@@ -934,10 +784,7 @@ static int launch_one(const Launch& l, FrontArgs<T> args, int nb, bool want_clus
       int max_clusters = 0;
       if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg) == cudaSuccess && max_clusters > 0) {
         const int groups = (nb + kCluster - 1) / kCluster;
-        const int own = groups < (owners + kCluster - 1) / kCluster ? groups : (owners + kCluster - 1) / kCluster;
-        int clusters = groups < max_clusters ? groups : max_clusters;
-        if (helpers && max_clusters > own) clusters = max_clusters;  // every SM that can hold a block streams
-        split_roles(args, clusters, own, helpers);
+        const int clusters = groups < max_clusters ? groups : max_clusters;
         cfg.gridDim = dim3(clusters * kCluster);
         const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, args);
         ++g_launch_count;
@@ -954,10 +801,7 @@ static int launch_one(const Launch& l, FrontArgs<T> args, int nb, bool want_clus
     (void)cudaGetLastError();
     return B2_STATUS_LAUNCH_FAILED;
   }
-  const int own = nb < owners ? nb : owners;
-  int grid = nb < sm_count() ? nb : sm_count();
-  if (helpers && sm_count() > own) grid = sm_count();
-  split_roles(args, grid, own, helpers);
+  const int grid = nb < sm_count() ? nb : sm_count();
   kern<<<grid, kT, smem, l.stream>>>(args);
   return check_launch();
 }
@@ -983,7 +827,7 @@ int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int6
   const int64_t nb64 = (n + NB - 1) / NB;
   if (nb64 > 0x3fffffff) return B2_STATUS_OK;
   const int nb = (int)nb64;
-  const int grid = sm_count();
+  const int grid = nb < sm_count() ? nb : sm_count();
   const size_t xbuf_words = (size_t)nb * NB * WPE;
   if (xbuf_words * 8 > l.scratch_bytes) return B2_STATUS_OK;
   FrontArgs<T> args = {};
@@ -995,34 +839,16 @@ int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int6
   args.xbuf = reinterpret_cast<unsigned long long*>(l.scratch);
   args.ctl = l.ctl;
   args.nb = nb;
+  {  // keep the prefetched-but-unused tiles of all blocks within a fraction of L2
+    const int64_t tile_bytes = (int64_t)NB * NB * sizeof(T);
+    int64_t d = knob(kKnobTrsvPrefetchBytes) / (tile_bytes * grid);
+    args.pf_dist = (int)(d < 0 ? 0 : d > 16 ? 16 : d);
+  }
   args.tag = tag;
   args.wait_limit = l.wait_limit;
   args.device_status = l.device_status;
   args.debug_skip = (int)knob(kKnobTrsvDebugSkip);
   args.pm_from = (int)knob(kKnobTrsvPmFrom);
-  {  // helper units, when the rows are long enough to have any and their partials fit the workspace
-    int near_min = (int)knob(kKnobTrsvHelpNear), chunk = (int)knob(kKnobTrsvHelpChunk);
-    if (near_min > 0 && near_min < 4) near_min = 4;
-    if (chunk < 2) chunk = 2;
-    chunk &= ~1;
-    const Units units = {(long long)nb - chunk - near_min, chunk, near_min};
-    const long long total = near_min > 0 ? units.total() : 0;
-    const size_t xbuf_bytes = (xbuf_words * 8 + 255) / 256 * 256;
-    if (total > 0 && total < 0x7fffffffLL && xbuf_bytes + (size_t)total * NB * WPE * 8 <= l.scratch_bytes) {
-      args.near_min = near_min;
-      args.chunk = chunk;
-      args.n_units = (unsigned)total;
-      args.hp = reinterpret_cast<unsigned long long*>(l.scratch + xbuf_bytes);
-    } else {
-      args.chunk = chunk;
-    }
-  }
-  {  // keep the prefetched-but-unused tiles of all blocks within a fraction of L2
-    const int64_t tile_bytes = (int64_t)NB * NB * sizeof(T);
-    const int busy = args.n_units > 0 ? grid : (nb < grid ? nb : grid);  // blocks that stream
-    int64_t d = knob(kKnobTrsvPrefetchBytes) / (tile_bytes * busy);
-    args.pf_dist = (int)(d < 0 ? 0 : d > 16 ? 16 : d);
-  }
   *handled = true;
   // (measured at n = 11520 / 8192: block by block with the premultiplied last tile is the
   // fastest form for both precisions -- float 156-162 us against 168-175 us in clusters of 8,

@@ -217,21 +217,17 @@ def test_trsv_bounded_wait_reports_timeout(b2):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
-@pytest.mark.parametrize("front,cluster,near,chunk", [(0, 0, 12, 8), (2, 0, 0, 8), (2, 2, 0, 8), (2, 0, 4, 2),
-                                                      (2, 2, 4, 2), (2, 0, 5, 4)])
-def test_trsv_every_kernel_choice(b2, ctx, dtype, front, cluster, near, chunk):
-    """trsv has three code paths (block-row kernel; sub-block kernel block by block, which
-    premultiplies the last tile; sub-block kernel in clusters), and the sub-block kernel runs with
-    or without helper blocks that take the far tiles of long rows.  The defaults pick one per
-    precision, view and size; here each is forced for every view, on sizes with a ragged last
-    block and more block rows than one cluster holds, with helper units small enough that these
-    sizes have several per row."""
-    old = (b2.get_tuning(b2.KNOB_TRSV_FRONT), b2.get_tuning(b2.KNOB_TRSV_CLUSTER),
-           b2.get_tuning(b2.KNOB_TRSV_HELP_NEAR), b2.get_tuning(b2.KNOB_TRSV_HELP_CHUNK))
+@pytest.mark.parametrize("front,cluster,pm_from", [(0, 0, 16), (2, 0, 0), (2, 0, 5), (2, 2, 0), (2, 2, 3)])
+def test_trsv_every_kernel_choice(b2, ctx, dtype, front, cluster, pm_from):
+    """trsv has three code paths (block-row kernel; sub-block kernel block by block; sub-block
+    kernel in clusters), and the sub-block kernel premultiplies the last tile of a block row from
+    a given row on.  The defaults pick one per precision and view; here each is forced for every
+    view, on sizes with a ragged last block and more block rows than one cluster holds, with the
+    premultiplied tile starting at the first row and inside the matrix."""
+    old = (b2.get_tuning(b2.KNOB_TRSV_FRONT), b2.get_tuning(b2.KNOB_TRSV_CLUSTER), b2.get_tuning(b2.KNOB_TRSV_PM_FROM))
     b2.set_tuning(b2.KNOB_TRSV_FRONT, front)
     b2.set_tuning(b2.KNOB_TRSV_CLUSTER, cluster)
-    b2.set_tuning(b2.KNOB_TRSV_HELP_NEAR, near)
-    b2.set_tuning(b2.KNOB_TRSV_HELP_CHUNK, chunk)
+    b2.set_tuning(b2.KNOB_TRSV_PM_FROM, pm_from)
     try:
         tol = TOL[np.dtype(dtype)]
         for n in (130, 1100, 2052):
@@ -248,8 +244,7 @@ def test_trsv_every_kernel_choice(b2, ctx, dtype, front, cluster, near, chunk):
     finally:
         b2.set_tuning(b2.KNOB_TRSV_FRONT, old[0])
         b2.set_tuning(b2.KNOB_TRSV_CLUSTER, old[1])
-        b2.set_tuning(b2.KNOB_TRSV_HELP_NEAR, old[2])
-        b2.set_tuning(b2.KNOB_TRSV_HELP_CHUNK, old[3])
+        b2.set_tuning(b2.KNOB_TRSV_PM_FROM, old[2])
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
@@ -374,8 +369,9 @@ def test_symv_trmv_every_unit_length(b2, ctx, dtype, unit):
     chosen by the matrix size; here each length is forced on sizes small enough for the full oracle
     and large enough to have rows of several units, a ragged edge, units of a single tile next to
     full ones, and several units per block (more units than SMs)."""
-    old = b2.get_tuning(b2.KNOB_TRI_TILE_UNIT)
+    old = b2.get_tuning(b2.KNOB_TRI_TILE_UNIT), b2.get_tuning(b2.KNOB_TRI_TILE)
     b2.set_tuning(b2.KNOB_TRI_TILE_UNIT, unit)
+    b2.set_tuning(b2.KNOB_TRI_TILE, 2)  # every trmv through the tile kernel too
     try:
         for n in (700, 2443):
             a = synth.matrix_np(17, 3, n, n, n, dtype, tri_n=n).ravel()
@@ -394,4 +390,32 @@ def test_symv_trmv_every_unit_length(b2, ctx, dtype, unit):
                     absterms = orc.trmv(orc.ROW_MAJOR, uplo, trans, diag, n, a, n, ox, 1)
                     assert_close(gx.host(), ox, absterms, dtype, f"trmv n={n} {uplo} {trans} {diag} unit={unit}")
     finally:
-        b2.set_tuning(b2.KNOB_TRI_TILE_UNIT, old)
+        b2.set_tuning(b2.KNOB_TRI_TILE_UNIT, old[0])
+        b2.set_tuning(b2.KNOB_TRI_TILE, old[1])
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("order", ORDERS)
+def test_trmv_tile_kernel_forced(b2, ctx, dtype, order):
+    """trmv through the shared-memory-ring tile kernel for every option combination (by default
+    only the cases where it is the faster one take it): padded leading dimension, strided and
+    reversed x, guard bands, the unreferenced triangle and a unit diagonal NaN-poisoned."""
+    old = b2.get_tuning(b2.KNOB_TRI_TILE)
+    b2.set_tuning(b2.KNOB_TRI_TILE, 2)
+    try:
+        for n, (pad, inc) in itertools.product((129, 700), ((0, 1), (4, 2), (8, -1))):
+            lda = n + pad
+            for uplo, trans, diag in itertools.product(UPLOS, TRANSES, DIAGS):
+                a = tri_buf(12, n, lda, dtype, order, uplo, diag)
+                x = synth.vector_np(7, n, n, dtype)
+                hx = place(x, inc)
+                ga, gx = Guarded(a), Guarded(hx)
+                b2.trmv(ctx, order, uplo, trans, diag, n, ga.t, lda, gx.t, inc)
+                ox = hx.copy()
+                absterms = orc.trmv(order, uplo, trans, diag, n, a, lda, ox, inc)
+                rx = gx.host()
+                assert_close(pick(rx, n, inc), pick(ox, n, inc), absterms, dtype, f"trmv n={n} pad={pad} inc={inc}")
+                assert_same_gaps(rx, hx, n, inc)
+                ga.check_guards(), gx.check_guards()
+    finally:
+        b2.set_tuning(b2.KNOB_TRI_TILE, old)
