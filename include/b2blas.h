@@ -92,6 +92,17 @@ int b2_version(void);
 /* Number of kernels this library has launched in this process so far (not thread-safe). */
 unsigned long long b2_launch_count(void);
 
+/* Bounds-checking build of the library (compiled with -DB2_DEBUG_BOUNDS into a separate file; no
+ * counterpart in the paper: it stands in for a memory checker).  In that build every kernel
+ * tests the addresses it touches against the extents of the call's arguments; an access
+ * outside them is skipped and counted, nothing traps.  b2_debug_bounds_report synchronises the
+ * device and writes {violations since the last report, first offending address, its size in
+ * bytes} to out3 (host memory).  b2_debug_bounds_shrink(bytes) is the checker's own test hook:
+ * it cuts `bytes` off the end of every extent, so that accesses which are in fact in bounds are
+ * reported.  Both return B2_STATUS_NOT_IMPLEMENTED in the ordinary build.  Not thread-safe. */
+int b2_debug_bounds_report(unsigned long long* out3);
+int b2_debug_bounds_shrink(int bytes);
+
 /* Tuning hooks (process-wide, not thread-safe): work-splitting parameters of the kernels,
  * indexed by the Knob enumeration of the sources.  Defaults are the tuned values; changing
  * them never changes what a routine computes, only how the work is cut.

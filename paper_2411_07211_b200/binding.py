@@ -31,7 +31,8 @@ KNOB_TRSV_PREFETCH_BYTES = 8
 KNOB_TRSV_FRONT, KNOB_TRSV_CLUSTER = 9, 10
 KNOB_TRSV_PM_FROM, KNOB_TRI_TILE, KNOB_TRI_TILE_UNIT = 11, 12, 13
 
-LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libb2blas.so")
+# B2BLAS_LIB selects another build of the same library (the bounds-checking one, libb2blas_dbg.so)
+LIB_PATH = os.environ.get("B2BLAS_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libb2blas.so")
 
 _i64, _int, _vp, _f, _d = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_float, ctypes.c_double
 
@@ -104,13 +105,18 @@ def lib():
         h.b2_set_tuning.restype = _int
         h.b2_get_tuning.argtypes = [_int]
         h.b2_get_tuning.restype = _i64
+        h.b2_debug_bounds_report.argtypes = [ctypes.POINTER(ctypes.c_ulonglong)]
+        h.b2_debug_bounds_report.restype = _int
+        h.b2_debug_bounds_shrink.argtypes = [_int]
+        h.b2_debug_bounds_shrink.restype = _int
         _lib = h
     return _lib
 
 
 def exported_symbols():
     return sorted(_protos().keys()) + ["b2_workspace_min_bytes", "b2_workspace_bytes", "b2_workspace_query", "b2_status_string",
-                                       "b2_version", "b2_launch_count", "b2_set_tuning", "b2_get_tuning"]
+                                       "b2_version", "b2_launch_count", "b2_set_tuning", "b2_get_tuning",
+                                       "b2_debug_bounds_report", "b2_debug_bounds_shrink"]
 
 
 class Context:
@@ -263,6 +269,23 @@ def set_tuning(knob: int, value: int):
 
 def get_tuning(knob: int) -> int:
     return int(lib().b2_get_tuning(knob))
+
+
+def debug_bounds_report():
+    """(violations since the last report, first offending address, its size) of the bounds-checking
+    build; None in the ordinary build."""
+    out = (ctypes.c_ulonglong * 3)()
+    st = lib().b2_debug_bounds_report(out)
+    if st == STATUS_NOT_IMPLEMENTED:
+        return None
+    if st:
+        raise B2Error("b2_debug_bounds_report", st)
+    return int(out[0]), int(out[1]), int(out[2])
+
+
+def debug_bounds_shrink(nbytes: int) -> bool:
+    """Test hook of the bounds-checking build; False in the ordinary build."""
+    return lib().b2_debug_bounds_shrink(int(nbytes)) == 0
 
 
 def launch_count() -> int:

@@ -22,6 +22,16 @@ static int64_t g_knobs[kKnobCount] = {
 
 unsigned long long g_launch_count = 0;
 
+#ifdef B2_DEBUG_BOUNDS
+static int g_dbg_shrink = 0;
+static void (*g_dbg_collectors[32])(unsigned long long*);
+static int g_dbg_ncollectors = 0;
+int dbg_shrink() { return g_dbg_shrink; }
+void dbg_register_collector(void (*fn)(unsigned long long*)) {
+  if (g_dbg_ncollectors < 32) g_dbg_collectors[g_dbg_ncollectors++] = fn;
+}
+#endif
+
 int64_t knob(int id) { return (id >= 0 && id < kKnobCount) ? g_knobs[id] : 0; }
 
 int sm_count() {
@@ -78,6 +88,29 @@ const char* b2_status_string(int status) {
     case B2_STATUS_BAD_CONTEXT: return "bad context (NULL, or workspace NULL / not 256-byte aligned)";
     default: return "unknown status";
   }
+}
+
+int b2_debug_bounds_report(unsigned long long* out3) {
+#ifdef B2_DEBUG_BOUNDS
+  if (out3 == nullptr) return -1;
+  if (cudaDeviceSynchronize() != cudaSuccess) return B2_STATUS_LAUNCH_FAILED;
+  out3[0] = out3[1] = out3[2] = 0;
+  for (int i = 0; i < b2::g_dbg_ncollectors; ++i) b2::g_dbg_collectors[i](out3);
+  return B2_STATUS_OK;
+#else
+  (void)out3;
+  return B2_STATUS_NOT_IMPLEMENTED;
+#endif
+}
+
+int b2_debug_bounds_shrink(int bytes) {
+#ifdef B2_DEBUG_BOUNDS
+  b2::g_dbg_shrink = bytes < 0 ? 0 : bytes;
+  return B2_STATUS_OK;
+#else
+  (void)bytes;
+  return B2_STATUS_NOT_IMPLEMENTED;
+#endif
 }
 
 int b2_version(void) { return 100; }

@@ -12,6 +12,53 @@
 
 namespace b2 {
 
+// ---------------------------------------------------------------------------------------
+// Bounds-checking build (-DB2_DEBUG_BOUNDS; a separate library file, never the default).  Every
+// entry point lists the byte ranges its kernels may touch (vector spans, matrix extents, result
+// words, the workspace); the load / store helpers and intrinsics below then test each address
+// against the list.  An access outside every range is NOT performed (a load gives zero): the
+// kernel records a count, the first offending address and its size in a report the host can
+// read, and carries on -- nothing traps, the context stays usable.
+#ifdef B2_DEBUG_BOUNDS
+struct DbgTable {
+  unsigned long long lo[8], hi[8];
+  int n;
+  int shrink;  // test hook: bytes cut off the end of every range (makes in-bounds accesses look bad)
+};
+struct DbgReport {
+  unsigned long long count, first_addr, first_bytes, pad;
+};
+static __device__ DbgTable g_dbg_table;    // one copy per translation unit, written before its kernels run
+static __device__ DbgReport g_dbg_report;  // accumulated until the host collects it
+__device__ __forceinline__ bool dbg_ok(const void* p, size_t bytes) {
+  const unsigned long long a = (unsigned long long)p;
+  for (int i = 0; i < g_dbg_table.n; ++i)
+    if (a >= g_dbg_table.lo[i] && a + bytes <= g_dbg_table.hi[i] - (unsigned long long)g_dbg_table.shrink) return true;
+  if (atomicAdd(&g_dbg_report.count, 1ull) == 0ull) {
+    g_dbg_report.first_addr = a;
+    g_dbg_report.first_bytes = bytes;
+  }
+  return false;
+}
+template <typename T>
+__device__ __forceinline__ T dbg_ldg(const T* p) { return dbg_ok(p, sizeof(T)) ? __ldg(p) : T(); }
+template <typename T>
+__device__ __forceinline__ T dbg_ldcg(const T* p) { return dbg_ok(p, sizeof(T)) ? __ldcg(p) : T(); }
+template <typename T>
+__device__ __forceinline__ T dbg_ldcs(const T* p) { return dbg_ok(p, sizeof(T)) ? __ldcs(p) : T(); }
+template <typename T>
+__device__ __forceinline__ void dbg_stcs(T* p, T v) { if (dbg_ok(p, sizeof(T))) __stcs(p, v); }
+#define __ldg(p) ::b2::dbg_ldg(p)
+#define __ldcg(p) ::b2::dbg_ldcg(p)
+#define __ldcs(p) ::b2::dbg_ldcs(p)
+#define __stcs(p, v) ::b2::dbg_stcs(p, v)
+#define B2_GUARD(p, bytes) ::b2::dbg_ok(p, bytes)
+#else
+#define B2_GUARD(p, bytes) true
+#endif
+// A plain store of a result element (checked in the bounds-checking build).
+#define B2_STORE(ptr, value) do { if (B2_GUARD(ptr, sizeof(*(ptr)))) *(ptr) = (value); } while (0)
+
 constexpr int kThreads = 256;  // every kernel uses 256-thread blocks (8 warps)
 constexpr int kWarps = kThreads / 32;
 
@@ -43,7 +90,8 @@ struct alignas(sizeof(T) * N) Pack {
 // Streaming (evict-first) load of data that may be written later by this kernel.
 template <typename T, int N>
 __device__ __forceinline__ Pack<T, N> ld_cs(const T* p) {
-  Pack<T, N> r;
+  Pack<T, N> r = {};
+  if (!B2_GUARD(p, sizeof(T) * N)) return r;
   if constexpr (sizeof(T) * N == 16) {
     uint4 t = __ldcs(reinterpret_cast<const uint4*>(p));
     r = *reinterpret_cast<Pack<T, N>*>(&t);
@@ -58,7 +106,8 @@ __device__ __forceinline__ Pack<T, N> ld_cs(const T* p) {
 // that the line is still there when the store arrives (see ld_cs for the evict-first form).
 template <typename T, int N>
 __device__ __forceinline__ Pack<T, N> ld_cg(const T* p) {
-  Pack<T, N> r;
+  Pack<T, N> r = {};
+  if (!B2_GUARD(p, sizeof(T) * N)) return r;
   if constexpr (sizeof(T) * N == 16) {
     uint4 t = __ldcg(reinterpret_cast<const uint4*>(p));
     r = *reinterpret_cast<Pack<T, N>*>(&t);
@@ -73,7 +122,8 @@ __device__ __forceinline__ Pack<T, N> ld_cg(const T* p) {
 // allocation so the matrix stream does not evict the reused vectors.
 template <typename T, int N>
 __device__ __forceinline__ Pack<T, N> ld_nc(const T* p) {
-  Pack<T, N> r;
+  Pack<T, N> r = {};
+  if (!B2_GUARD(p, sizeof(T) * N)) return r;
   if constexpr (sizeof(T) * N == 16) {
     uint4 t;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -90,7 +140,8 @@ __device__ __forceinline__ Pack<T, N> ld_nc(const T* p) {
 // Read-only load of reused data (the x vectors): cached in L1.
 template <typename T, int N>
 __device__ __forceinline__ Pack<T, N> ld_ro(const T* p) {
-  Pack<T, N> r;
+  Pack<T, N> r = {};
+  if (!B2_GUARD(p, sizeof(T) * N)) return r;
   if constexpr (sizeof(T) * N == 16) {
     uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
     r = *reinterpret_cast<Pack<T, N>*>(&t);
@@ -103,6 +154,7 @@ __device__ __forceinline__ Pack<T, N> ld_ro(const T* p) {
 
 template <typename T, int N>
 __device__ __forceinline__ void st_cs(T* p, const Pack<T, N>& r) {
+  if (!B2_GUARD(p, sizeof(T) * N)) return;
   if constexpr (sizeof(T) * N == 16) {
     __stcs(reinterpret_cast<uint4*>(p), *reinterpret_cast<const uint4*>(&r));
   } else {
@@ -174,6 +226,10 @@ struct Launch {
   unsigned* ctl;         // control block as 32-bit words
   int* device_status;
   unsigned long long wait_limit;
+#ifdef B2_DEBUG_BOUNDS
+  unsigned long long dbg_lo[8], dbg_hi[8];  // byte ranges the kernels of this call may touch
+  int dbg_n;
+#endif
 };
 
 inline int make_launch(const b2_ctx* ctx, Launch* l) {
@@ -186,6 +242,9 @@ inline int make_launch(const b2_ctx* ctx, Launch* l) {
   l->scratch_bytes = ctx->workspace_bytes - kCtlBytes;
   l->device_status = ctx->device_status;
   l->wait_limit = ctx->wait_limit;
+#ifdef B2_DEBUG_BOUNDS
+  l->dbg_n = 0;
+#endif
   return B2_STATUS_OK;
 }
 
@@ -195,6 +254,54 @@ inline int check_launch() {
   ++g_launch_count;
   return cudaGetLastError() == cudaSuccess ? B2_STATUS_OK : B2_STATUS_LAUNCH_FAILED;
 }
+
+// Bounds-checking build: the ranges a call may touch, and their hand-over to this translation
+// unit's device table (stream-ordered, before the kernels of the call).  No-ops otherwise.
+#ifdef B2_DEBUG_BOUNDS
+int dbg_shrink();  // test hook value (bytes)
+void dbg_register_collector(void (*fn)(unsigned long long*));
+inline void dbg_range(Launch& l, const void* p, size_t bytes) {
+  if (p == nullptr || bytes == 0 || l.dbg_n >= 8) return;
+  l.dbg_lo[l.dbg_n] = (unsigned long long)p;
+  l.dbg_hi[l.dbg_n] = (unsigned long long)p + bytes;
+  ++l.dbg_n;
+}
+template <typename T>
+inline void dbg_vec(Launch& l, const T* p, int64_t n, int64_t inc) {  // p as the caller passes it
+  if (n <= 0) return;
+  const int64_t span = 1 + (n - 1) * (inc < 0 ? -inc : inc);
+  dbg_range(l, p, (size_t)span * sizeof(T));
+}
+static void dbg_collect_this_unit(unsigned long long* out) {
+  DbgReport r = {};
+  if (cudaMemcpyFromSymbol(&r, g_dbg_report, sizeof(r)) != cudaSuccess) return;
+  if (r.count && out[0] == 0) out[1] = r.first_addr, out[2] = r.first_bytes;
+  out[0] += r.count;
+  const DbgReport zero = {};
+  cudaMemcpyToSymbol(g_dbg_report, &zero, sizeof(zero));
+}
+static void dbg_commit(Launch& l) {
+  static bool registered = false;  // (one flag per translation unit, like the device symbols)
+  if (!registered) {
+    registered = true;
+    dbg_register_collector(&dbg_collect_this_unit);
+  }
+  dbg_range(l, l.ctl, kCtlBytes + l.scratch_bytes);  // the workspace, whole
+  DbgTable t = {};
+  for (int i = 0; i < l.dbg_n && i < 8; ++i) t.lo[i] = l.dbg_lo[i], t.hi[i] = l.dbg_hi[i];
+  t.n = l.dbg_n < 8 ? l.dbg_n : 8;
+  t.shrink = dbg_shrink();
+  cudaMemcpyToSymbolAsync(g_dbg_table, &t, sizeof(t), 0, cudaMemcpyHostToDevice, l.stream);
+  --l.dbg_n;  // (a second commit of the same call adds the workspace again)
+}
+#define B2_DBG_VEC(l, p, n, inc) ::b2::dbg_vec(l, p, n, inc)
+#define B2_DBG_RANGE(l, p, bytes) ::b2::dbg_range(l, p, bytes)
+#define B2_DBG_COMMIT(l) ::b2::dbg_commit(l)
+#else
+#define B2_DBG_VEC(l, p, n, inc) ((void)0)
+#define B2_DBG_RANGE(l, p, bytes) ((void)0)
+#define B2_DBG_COMMIT(l) ((void)0)
+#endif
 
 // Number of SMs of the current device (cached per device id).
 int sm_count();

@@ -27,6 +27,10 @@ static int gemv_impl(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t
   Launch l;
   if (int st = make_launch(ctx, &l)) return st;
   if (m == 0 || n == 0) return B2_STATUS_OK;
+  B2_DBG_RANGE(l, a, (size_t)(((order == B2_ROW_MAJOR ? m : n) - 1) * lda + minor) * sizeof(T));
+  B2_DBG_VEC(l, x, lenx, incx);
+  B2_DBG_VEC(l, y, leny, incy);
+  B2_DBG_COMMIT(l);
   if (alpha == T(0)) return scale_y<T>(l, y, incy, leny, beta);
 
   L2Args<T> args = {};

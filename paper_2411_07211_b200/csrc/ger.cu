@@ -134,6 +134,10 @@ static int ger_impl(const b2_ctx* ctx, int order, int64_t m, int64_t n, T alpha,
   Launch l;
   if (int st = make_launch(ctx, &l)) return st;
   if (m == 0 || n == 0 || alpha == T(0)) return B2_STATUS_OK;
+  B2_DBG_RANGE(l, a, (size_t)(((order == B2_ROW_MAJOR ? m : n) - 1) * lda + minor) * sizeof(T));
+  B2_DBG_VEC(l, x, m, incx);
+  B2_DBG_VEC(l, y, n, incy);
+  B2_DBG_COMMIT(l);
   // canonical row-major view: row vector index = slow dimension of the buffer
   const bool rm = order == B2_ROW_MAJOR;
   const int64_t rows = rm ? m : n, cols = rm ? n : m;

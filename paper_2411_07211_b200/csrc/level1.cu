@@ -547,6 +547,9 @@ static int run_map(const b2_ctx* ctx, Op op, int64_t n, T* x, int64_t incx, T* y
   if (n == 0) return B2_STATUS_OK;
   constexpr bool two = Op::RY || Op::WY;
   constexpr int V = VecLen<T>::value;
+  B2_DBG_VEC(l, x, n, incx);
+  if (two) B2_DBG_VEC(l, y, n, incy);
+  B2_DBG_COMMIT(l);
   int64_t head = 0;
   if (incx == 1 && (!two || incy == 1) && same_head<T>(x, y, two, &head)) {
     constexpr int NV = two ? 4 : 8;
@@ -577,6 +580,10 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
   }
   constexpr int V = VecLen<T>::value;
   if (n > ((int64_t)1 << 40)) return B2_STATUS_NOT_IMPLEMENTED;  // chunk ids are 32-bit
+  B2_DBG_VEC(l, x, n, incx);
+  if (Op::RY) B2_DBG_VEC(l, y, n, incy);
+  B2_DBG_RANGE(l, result, sizeof(typename Op::Out));
+  B2_DBG_COMMIT(l);
   const int cap = grid_cap();
   if (l.scratch_bytes < (size_t)cap * sizeof(Acc)) return B2_STATUS_WORKSPACE_TOO_SMALL;
   Acc* partials = reinterpret_cast<Acc*>(l.scratch);

@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args
       if (q % LPV == 0 && i < r_end) {
         if (p.direct) {
           T* yp = p.y + i * p.incy;
-          *yp = p.beta != T(0) ? p.alpha * s + p.beta * *yp : p.alpha * s;
+          B2_STORE(yp, p.beta != T(0) ? p.alpha * s + p.beta * *yp : p.alpha * s);
         } else {
           p.rowpart[(int64_t)cs * p.rows + i] = s;
         }
@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args
       for (int w = 1; w < kWarps; ++w) s += sm[w][t];
       if (p.direct) {
         T* yp = p.y + j * p.incy;
-        *yp = p.beta != T(0) ? p.alpha * s + p.beta * *yp : p.alpha * s;
+        B2_STORE(yp, p.beta != T(0) ? p.alpha * s + p.beta * *yp : p.alpha * s);
       } else {
         p.colpart[rs * p.cols + j] = s;
       }
@@ -347,7 +347,7 @@ __global__ void __launch_bounds__(kThreads) l2_finalize(const L2Args<T> p, int R
   }
   if (i < nout) {
     T* yp = p.y + i * p.incy;
-    *yp = p.beta != T(0) ? p.alpha * s + p.beta * *yp : p.alpha * s;
+    B2_STORE(yp, p.beta != T(0) ? p.alpha * s + p.beta * *yp : p.alpha * s);
   }
 }
 

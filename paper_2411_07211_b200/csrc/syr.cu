@@ -192,6 +192,10 @@ static int syr_impl(const b2_ctx* ctx, int order, int uplo, int64_t n, T alpha, 
   Launch l;
   if (int st = make_launch(ctx, &l)) return st;
   if (n == 0 || alpha == T(0)) return B2_STATUS_OK;
+  B2_DBG_RANGE(l, a, (size_t)((n - 1) * lda + n) * sizeof(T));
+  B2_DBG_VEC(l, x, n, incx);
+  if (TWO) B2_DBG_VEC(l, y, n, incy);
+  B2_DBG_COMMIT(l);
   // canonical row-major view: a column-major upper triangle is a row-major lower one; the
   // update itself is symmetric in (i, j), so nothing else changes
   const bool lower = (uplo == B2_LOWER) == (order == B2_ROW_MAJOR);

@@ -44,6 +44,10 @@ static int symv_impl(const b2_ctx* ctx, int order, int uplo, int64_t n, T alpha,
   Launch l;
   if (int st = make_launch(ctx, &l)) return st;
   if (n == 0) return B2_STATUS_OK;
+  B2_DBG_RANGE(l, a, (size_t)((n - 1) * lda + n) * sizeof(T));
+  B2_DBG_VEC(l, x, n, incx);
+  B2_DBG_VEC(l, y, n, incy);
+  B2_DBG_COMMIT(l);
   if (alpha == T(0)) return scale_y<T>(l, y, incy, n, beta);
   L2Args<T> args = {};
   args.a = a;
@@ -101,6 +105,9 @@ static int trmv_impl(const b2_ctx* ctx, int order, int uplo, int trans, int diag
   Launch l;
   if (int st = make_launch(ctx, &l)) return st;
   if (n == 0) return B2_STATUS_OK;
+  B2_DBG_RANGE(l, a, (size_t)((n - 1) * lda + n) * sizeof(T));
+  B2_DBG_VEC(l, x, n, incx);
+  B2_DBG_COMMIT(l);
   L2Args<T> args = {};
   args.a = a;
   args.lda = lda;

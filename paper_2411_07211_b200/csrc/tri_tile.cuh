@@ -83,15 +83,21 @@ __host__ __device__ __forceinline__ void col_range(int J, int64_t n, int nbr, in
 // Asynchronous 16-byte copy global -> shared memory of `bytes` (0 .. 16) bytes, the rest of the
 // 16 zero-filled; element-sized copies for the vectors (bytes = 0: a zero).
 __device__ __forceinline__ void cp_async16_full(void* dst, const void* src) {
+  if (!B2_GUARD(src, 16)) {  // (bounds-checking build only: a zero-filled pack instead of the read)
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, 0;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+    return;
+  }
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async16(void* dst, const void* src, int bytes) {
+  if (bytes > 0 && !B2_GUARD(src, (size_t)bytes)) bytes = 0;
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src),
                "r"(bytes)
                : "memory");
 }
 template <int N>
 __device__ __forceinline__ void cp_async_elem(void* dst, const void* src, bool valid) {
+  if (valid && !B2_GUARD(src, (size_t)N)) valid = false;
   asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src),
                "n"(N), "r"(valid ? N : 0)
                : "memory");
@@ -392,7 +398,7 @@ __global__ void __launch_bounds__(fin_warps<T>() * 32) tri_tile_finalize(const T
 #pragma unroll
     for (int k = 1; k < kFinWarps; ++k) t += part[k][lane];
     T* yp = p.y + i * p.incy;
-    *yp = p.beta != T(0) ? p.alpha * t + p.beta * *yp : p.alpha * t;
+    B2_STORE(yp, p.beta != T(0) ? p.alpha * t + p.beta * *yp : p.alpha * t);
   }
 }
 

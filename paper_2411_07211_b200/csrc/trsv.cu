@@ -404,7 +404,9 @@ __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
 #pragma unroll
       for (int j = 0; j < EPL; ++j) {
         const int el = lane * EPL + j, t = el / kSB, lc = el % kSB;
-        xsm[((s + t) % kXB) * kSB + lc] = wp[j * WPE] ? decode(&w[j * WPE], T(0)) : T(0);
+        // (a tile past the end of the row has no buffer of its own: the slot it would map to may
+        // still be read by the compute warps, four tiles behind)
+        if (s + t < nsrc) xsm[((s + t) % kXB) * kSB + lc] = wp[j * WPE] ? decode(&w[j * WPE], T(0)) : T(0);
       }
       __threadfence_block();
 #pragma unroll
@@ -572,6 +574,9 @@ static int trsv_impl(const b2_ctx* ctx, int order, int uplo, int trans, int diag
   Launch l;
   if (int st = make_launch(ctx, &l)) return st;
   if (n == 0) return B2_STATUS_OK;
+  B2_DBG_RANGE(l, a, (size_t)((n - 1) * lda + n) * sizeof(T));
+  B2_DBG_VEC(l, x, n, incx);
+  B2_DBG_COMMIT(l);
   // op(A) lower triangular <=> forward substitution
   const bool eff_lower = (uplo == B2_LOWER) != (trans == B2_TRANS);
   // rows of op(A) contiguous in memory <=> row-major N or column-major T

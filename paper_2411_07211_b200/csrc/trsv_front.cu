@@ -850,6 +850,12 @@ int trsv_front_try(const Launch& l, bool coltype, bool backward, bool unit, int6
   args.debug_skip = (int)knob(kKnobTrsvDebugSkip);
   args.pm_from = (int)knob(kKnobTrsvPmFrom);
   *handled = true;
+#ifdef B2_DEBUG_BOUNDS
+  {  // (this translation unit has its own copy of the range table)
+    Launch lc = l;
+    B2_DBG_COMMIT(lc);
+  }
+#endif
   // (measured at n = 11520 / 8192: block by block with the premultiplied last tile is the
   // fastest form for both precisions -- float 156-162 us against 168-175 us in clusters of 8,
   // double 180 us against 216 us -- so clusters are off by default)
