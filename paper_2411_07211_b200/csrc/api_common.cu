@@ -18,6 +18,7 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobTrsvPmFrom      */ 16,
     /* kKnobTriTile         */ 1,
     /* kKnobTriTileUnit     */ 0,
+    /* kKnobNarrowBlock     */ 1,
 };
 
 unsigned long long g_launch_count = 0;

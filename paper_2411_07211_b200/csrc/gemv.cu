@@ -46,12 +46,39 @@ static int gemv_impl(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t
   if (rowdot) {
     args.xc = vec_base(x, lenx, incx);
     args.incxc = incx;
+    if (knob(kKnobNarrowBlock) && block_narrow_applies(a, lda, args.rows, args.cols))
+      return block_rowdot<T>(l, a, args.rows, args.cols, args.xc, incx, alpha, beta, args.y, incy);
     if (skinny_applies(a, lda, args.rows, args.cols, true))
       return skinny_rowdot<T>(l, a, args.rows, args.cols, args.xc, incx, alpha, beta, args.y, incy);
     return l2_dispatch<T, GemvRow, true>(l, args, plan_rowout(args, true), true);
   }
   args.xr = vec_base(x, lenx, incx);
   args.incxr = incx;
+  if (knob(kKnobNarrowBlock) && wide_applies<T>(args.rows, args.cols)) {
+    const int64_t want = (args.cols + kThreads - 1) / kThreads, cap = (int64_t)sm_count() * 8;
+    wide_colsum_kernel<T><<<(unsigned)(want < cap ? want : cap), kThreads, 0, l.stream>>>(a, lda, (int)args.rows, args.cols, args.xr,
+                                                                                   incx, alpha, beta, args.y, incy);
+    return check_launch();
+  }
+  if (knob(kKnobNarrowBlock) && block_narrow_applies(a, lda, args.rows, args.cols)) {
+    const int ppr = (int)(args.cols / VecLen<T>::value), K = kThreads / ppr;
+    const int64_t nsteps = (args.rows + (int64_t)K * kBlockUnroll - 1) / ((int64_t)K * kBlockUnroll);
+    const int64_t cap = (int64_t)sm_count() * 4;
+    const int grid = (int)(nsteps < cap ? nsteps : cap);
+    if ((size_t)grid * args.cols * sizeof(T) <= l.scratch_bytes) {
+      args.colpart = reinterpret_cast<T*>(l.scratch);
+      args.nrs = grid;  // one partial row per block; the finalize kernel adds all of them
+      args.ncs = 1;
+      args.nct = 1;
+      args.ctiles_per_cta = 1;
+      args.rows_per_cta = args.rows;
+      args.direct = 0;
+      block_colsum_kernel<T><<<grid, kThreads, 0, l.stream>>>(a, args.rows, ppr, args.xr, incx, args.colpart, nsteps);
+      if (int st = check_launch()) return st;
+      launch_finalize<T, GemvCol, 32>(l, args, 1, (int)args.cols, args.cols);
+      return check_launch();
+    }
+  }
   if (skinny_colsum_applies(a, lda, args.rows, args.cols)) {
     const int ppr = (int)(args.cols / VecLen<T>::value);
     const int64_t rows_per_step = (int64_t)(32 / ppr) * kColsumGroup;

@@ -146,6 +146,13 @@ static int ger_impl(const b2_ctx* ctx, int order, int64_t m, int64_t n, T alpha,
   const T* yc = rm ? vec_base(y, n, incy) : vec_base(x, m, incx);
   const int64_t incyc = rm ? incy : incx;
   constexpr int V = VecLen<T>::value;
+  // (measured: the element-wise walk wins in double; in float the pack kernels stay ahead)
+  if (knob(kKnobNarrowBlock) && sizeof(T) == 8 && wide_applies<T>(rows, cols)) {
+    const int64_t want = (cols + kThreads - 1) / kThreads, cap = (int64_t)sm_count() * 8;
+    wide_ger_kernel<T><<<(unsigned)(want < cap ? want : cap), kThreads, 0, l.stream>>>(a, lda, (int)rows, cols, xr, incxr, yc, incyc,
+                                                                                alpha);
+    return check_launch();
+  }
   if (skinny_applies(a, lda, rows, cols, false)) return skinny_ger<T>(l, a, rows, cols, xr, incxr, yc, incyc, alpha);
   if (aligned_to(a, 16) && lda % V == 0) return ger_shape<T, V>(l, a, lda, rows, cols, xr, incxr, yc, incyc, alpha);
   return ger_shape<T, 1>(l, a, lda, rows, cols, xr, incxr, yc, incyc, alpha);

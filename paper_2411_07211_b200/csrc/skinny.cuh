@@ -226,6 +226,198 @@ static bool skinny_colsum_applies(const T* a, int64_t lda, int64_t rows, int64_t
   return 100 * busy >= 100 * 32 * ppr / lanes + 15 * 32;
 }
 
+// Block-wide forms of the two gemv kinds for any row length up to kBlockMaxPpr packs: a row gets
+// exactly PPR THREADS of the block (not lanes of one warp), so K = 256 / PPR whole rows are one
+// contiguous run of K * PPR packs per step -- 240 of 256 threads at 20 packs per row, where a warp
+// on its own would use 20 of its 32 lanes.  A thread's column pack never changes: its slice of x
+// (row-dot) or its column sums (column kind) stay in registers.  kBlockUnroll steps are in flight.
+constexpr int kBlockMaxPpr = 64;
+constexpr int kBlockUnroll = 8;
+
+// y_i <- alpha * sum_j a_ij x_j + beta * y_i.  Per pack one partial; the PPR partials of a row meet
+// in shared memory (odd pitch), where one thread per row adds them in column order.
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 3) block_rowdot_kernel(const T* __restrict__ a, int64_t rows, int ppr,
+                                                                   const T* __restrict__ x, int64_t incx, T alpha,
+                                                                   T beta, T* __restrict__ y, int64_t incy,
+                                                                   int64_t nsteps) {
+  constexpr int V = VecLen<T>::value, U = kBlockUnroll;
+  using P = Pack<T, V>;
+  extern __shared__ __align__(16) unsigned char block_smem[];
+  T* part = reinterpret_cast<T*>(block_smem);  // [U][K * pitch]
+  const int t = (int)threadIdx.x, K = kThreads / ppr, G = K * ppr, pitch = ppr | 1;
+  const bool active = t < G;
+  const int c = t % ppr, r = t / ppr;
+  T xv[V];
+#pragma unroll
+  for (int e = 0; e < V; ++e) xv[e] = active ? __ldg(x + (int64_t)(c * V + e) * incx) : T(0);
+  const int64_t rows_per_step = (int64_t)K * U;
+  for (int64_t step = blockIdx.x; step < nsteps; step += gridDim.x) {
+    const int64_t row0 = step * rows_per_step;
+    const P* src = reinterpret_cast<const P*>(a) + row0 * ppr + t;
+    P av[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+#pragma unroll
+      for (int e = 0; e < V; ++e) av[u].v[e] = T(0);
+      if (active && row0 + u * K + r < rows) av[u] = ld_nc<T, V>(reinterpret_cast<const T*>(src + (int64_t)u * G));
+    }
+    if (active) {
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        T s = T(0);
+#pragma unroll
+        for (int e = 0; e < V; ++e) s = av[u].v[e] * xv[e] + s;
+        part[(u * K + r) * pitch + c] = s;
+      }
+    }
+    __syncthreads();
+    for (int j = t; j < K * U; j += kThreads) {
+      const int64_t row = row0 + j;  // (slot j = u * K + r holds row row0 + u * K + r)
+      if (row < rows) {
+        T s = T(0);
+        for (int q = 0; q < ppr; ++q) s += part[j * pitch + q];
+        T* yp = y + row * incy;
+        B2_STORE(yp, beta != T(0) ? alpha * s + beta * *yp : alpha * s);
+      }
+    }
+    __syncthreads();  // part is rewritten by the next step
+  }
+}
+
+// colpart[block][j] = sum over the block's rows of a_ij * x_i (the general finalize kernel adds
+// the blocks' rows in a fixed order and applies alpha / beta).
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 4) block_colsum_kernel(const T* __restrict__ a, int64_t rows, int ppr,
+                                                                   const T* __restrict__ xr, int64_t incxr,
+                                                                   T* __restrict__ colpart, int64_t nsteps) {
+  constexpr int V = VecLen<T>::value, U = kBlockUnroll;
+  using P = Pack<T, V>;
+  __shared__ T sm[kThreads * V];
+  grid_dep_launch();
+  const int t = (int)threadIdx.x, K = kThreads / ppr, G = K * ppr;
+  const bool active = t < G;
+  const int r = t / ppr;
+  const int64_t rows_per_step = (int64_t)K * U;
+  T acc[V];
+#pragma unroll
+  for (int e = 0; e < V; ++e) acc[e] = T(0);
+  for (int64_t step = blockIdx.x; step < nsteps; step += gridDim.x) {
+    const int64_t row0 = step * rows_per_step;
+    const P* src = reinterpret_cast<const P*>(a) + row0 * ppr + t;
+    P av[U];
+    T xv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int64_t row = row0 + u * K + r;
+      xv[u] = T(0);
+#pragma unroll
+      for (int e = 0; e < V; ++e) av[u].v[e] = T(0);
+      if (active && row < rows) {
+        av[u] = ld_nc<T, V>(reinterpret_cast<const T*>(src + (int64_t)u * G));
+        xv[u] = __ldg(xr + row * incxr);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int e = 0; e < V; ++e) acc[e] = av[u].v[e] * xv[u] + acc[e];
+  }
+  // threads rr * ppr + q (all rr) hold partial sums of column pack q
+#pragma unroll
+  for (int e = 0; e < V; ++e) sm[t * V + e] = active ? acc[e] : T(0);
+  __syncthreads();
+  for (int j = t; j < ppr * V; j += kThreads) {
+    const int q = j / V, e = j % V;
+    T s = T(0);
+    for (int rr = 0; rr < K; ++rr) s += sm[(rr * ppr + q) * V + e];
+    colpart[(int64_t)blockIdx.x * (ppr * V) + j] = s;
+  }
+}
+
+// The block-wide kernels apply to unpadded, 16-byte aligned matrices of many narrow rows.
+template <typename T>
+static bool block_narrow_applies(const T* a, int64_t lda, int64_t rows, int64_t cols) {
+  constexpr int V = VecLen<T>::value;
+  if (rows < kSkinnyMinRows || cols != lda || cols % V != 0 || !aligned_to(a, 16)) return false;
+  const int64_t ppr = cols / V;
+  return ppr >= 1 && ppr <= kBlockMaxPpr;
+}
+
+template <typename T>
+static int block_rowdot(const Launch& l, const T* a, int64_t rows, int64_t cols, const T* x, int64_t incx, T alpha,
+                        T beta, T* y, int64_t incy) {
+  const int ppr = (int)(cols / VecLen<T>::value), K = kThreads / ppr;
+  const int64_t nsteps = (rows + (int64_t)K * kBlockUnroll - 1) / ((int64_t)K * kBlockUnroll);
+  const int64_t cap = (int64_t)sm_count() * 3;
+  const size_t smem = sizeof(T) * (size_t)kBlockUnroll * K * (ppr | 1);
+  block_rowdot_kernel<T><<<(unsigned)(nsteps < cap ? nsteps : cap), kThreads, smem, l.stream>>>(a, rows, ppr, x, incx, alpha,
+                                                                                          beta, y, incy, nsteps);
+  return check_launch();
+}
+
+// The transposed shape: a canonical view of FEW (<= kWideMaxRows) very long rows -- what a narrow
+// column-major matrix looks like.  A thread owns columns and walks down the few rows, so every
+// load instruction of a warp is one contiguous run of a row whatever the alignment of the rows
+// (an odd leading dimension puts every second row off the 16-byte boundary: element loads do not
+// care), nothing is reduced across lanes, and x is staged once.  (The row-dot kind of this shape
+// stays on the general kernel: a column-owning form of it measured no faster.)
+constexpr int kWideMaxRows = 64;
+constexpr int64_t kWideMinCols = 1 << 15;
+
+template <typename T>
+static bool wide_applies(int64_t rows, int64_t cols) {
+  return rows >= 1 && rows <= kWideMaxRows && cols >= kWideMinCols;
+}
+
+// y_j <- alpha * sum_i a_ij x_i + beta * y_j (one output per column, written directly).
+template <typename T>
+__global__ void __launch_bounds__(kThreads) wide_colsum_kernel(const T* __restrict__ a, int64_t lda, int rows, int64_t cols,
+                                                               const T* __restrict__ xr, int64_t incxr, T alpha, T beta,
+                                                               T* __restrict__ y, int64_t incy) {
+  __shared__ T xs[kWideMaxRows];
+  if (threadIdx.x < rows) xs[threadIdx.x] = __ldg(xr + threadIdx.x * incxr);
+  __syncthreads();
+  for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < cols; j += (int64_t)gridDim.x * kThreads) {
+    const T* col = a + j;
+    T acc = T(0);
+    int i = 0;
+    for (; i + 8 <= rows; i += 8) {
+      T v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = __ldg(col + (int64_t)(i + k) * lda);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc = v[k] * xs[i + k] + acc;
+    }
+    for (; i < rows; ++i) acc = __ldg(col + (int64_t)i * lda) * xs[i] + acc;
+    T* yp = y + j * incy;
+    B2_STORE(yp, beta != T(0) ? alpha * acc + beta * *yp : alpha * acc);
+  }
+}
+
+// a_ij <- alpha * x_i * y_j + a_ij, x indexed by the few rows, y by the many columns.
+template <typename T>
+__global__ void __launch_bounds__(kThreads) wide_ger_kernel(T* __restrict__ a, int64_t lda, int rows, int64_t cols,
+                                                            const T* __restrict__ xr, int64_t incxr,
+                                                            const T* __restrict__ yc, int64_t incyc, T alpha) {
+  __shared__ T xs[kWideMaxRows];
+  if (threadIdx.x < rows) xs[threadIdx.x] = alpha * __ldg(xr + threadIdx.x * incxr);
+  __syncthreads();
+  for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < cols; j += (int64_t)gridDim.x * kThreads) {
+    T* col = a + j;
+    const T yj = __ldg(yc + j * incyc);
+    int i = 0;
+    for (; i + 8 <= rows; i += 8) {
+      T v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = __ldcg(col + (int64_t)(i + k) * lda);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) __stcs(col + (int64_t)(i + k) * lda, xs[i + k] * yj + v[k]);
+    }
+    for (; i < rows; ++i) __stcs(col + (int64_t)i * lda, xs[i] * yj + __ldcg(col + (int64_t)i * lda));
+  }
+}
+
 template <typename T>
 static int skinny_grid(int64_t nchunks) {
   const int64_t blocks = (nchunks + kWarps - 1) / kWarps;
