@@ -371,13 +371,16 @@ def configs_leg(device, peak: float, reps: int, only=None):
     rows = []
 
     def batch_ms(call, nbuf, count):
-        """Median over 5 batches of `count` calls (buffer k % nbuf), per call."""
+        """Median over 5 batches of `count` calls (buffer k % nbuf), per call.  The calls are
+        marshalled once (binding.prepare): a Python wrapper call costs more than a small kernel."""
+        fast = [b2.prepare(lambda k=k: call(k)) for k in range(nbuf)]
+        order = [fast[k % nbuf] for k in range(count)]
         ts = []
         for it in range(7):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            for k in range(count):
-                call(k % nbuf)
+            for f in order:
+                f()
             e1.record()
             torch.cuda.synchronize()
             if it >= 2:
@@ -422,13 +425,13 @@ def configs_leg(device, peak: float, reps: int, only=None):
 
     # ---- level 1: config 1 (sdot, 1 Mi floats) is the n = 2^20 row of the sweep
     for dt, s in (("f32", 4), ("f64", 8)):
-        pool = synth.vector_torch(0, 20, (768 * MIB) // s, tdt[dt], device)  # rotating sets are slices of this
+        pool = synth.vector_torch(0, 20, 1 << 29, tdt[dt], device)  # rotating sets are slices of this (2 GiB / 4 GiB)
         for lg in (16, 20, 24, 28):
             n = 1 << lg
             for inc in (1, 2):
                 span = n * inc
                 if 2 * span > pool.numel():
-                    continue  # (2^28 doubles with increment 2 would need 8 GiB for two vectors)
+                    continue  # (n = 2^28 with increment 2: two spans of 2^29 elements do not fit the pool)
                 res = torch.zeros(4, dtype=tdt[dt], device=device)
                 ires = torch.zeros(1, dtype=torch.int64, device=device)
                 for r, per_elem, nvec in (("axpy", 3, 2), ("scal", 2, 1), ("copy", 2, 2), ("swap", 4, 2),

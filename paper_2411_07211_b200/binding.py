@@ -166,12 +166,39 @@ def _prefix(t) -> str:
     raise TypeError(f"b2blas supports float32/float64, got {t.dtype}")
 
 
+_recording = None  # list of (function, ctx struct, args) while prepare() runs a thunk
+
+
 def _call(name, ctx: Context, *args, check=True):
     c = ctx.struct()
-    st = getattr(lib(), name)(ctypes.byref(c), *args)
+    fn = getattr(lib(), name)
+    st = fn(ctypes.byref(c), *args)
+    if _recording is not None:
+        _recording.append((fn, c, args))
     if check and st != 0:
         raise B2Error(name, st)
     return st
+
+
+def prepare(thunk):
+    """Runs `thunk` (calls of this module) once and returns a callable that repeats exactly those
+    library calls with the arguments marshalled then -- same stream, same pointers -- without the
+    per-call Python work of the wrappers (about 10 us a call, more than a small kernel takes).
+    For timing loops over small problems; the returned callable returns the last status."""
+    global _recording
+    _recording = rec = []
+    try:
+        thunk()
+    finally:
+        _recording = None
+    calls = [(fn, ctypes.byref(c), args, c) for fn, c, args in rec]
+
+    def replay():
+        st = 0
+        for fn, ref, args, _keep in calls:
+            st = fn(ref, *args)
+        return st
+    return replay
 
 
 # ---- level 1 ----------------------------------------------------------------------------
