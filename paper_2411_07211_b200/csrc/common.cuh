@@ -327,6 +327,27 @@ enum Knob {
 };
 int64_t knob(int id);
 
+// Launch with programmatic stream serialization: the grid may be scheduled while its predecessor
+// in the stream drains.  Every kernel launched this way starts with grid_dep_wait() (nothing
+// of the predecessor's memory is read or written before the predecessor has completed and
+// flushed) followed by grid_dep_launch() (its own successor may be scheduled as soon as all
+// of its blocks are resident), so the chain of completions stays transitive.
+template <typename... KArgs, typename... Args>
+inline void launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = knob(kKnobUsePdl) ? 1 : 0;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);  // (a failure is picked up by check_launch())
+}
+
+
 // Base pointer such that logical element i lives at base[i*inc] for either sign of inc.
 template <typename T>
 inline T* vec_base(T* p, int64_t n, int64_t inc) {

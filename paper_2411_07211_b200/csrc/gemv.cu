@@ -56,7 +56,7 @@ static int gemv_impl(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t
   args.incxr = incx;
   if (knob(kKnobNarrowBlock) && wide_applies<T>(args.rows, args.cols)) {
     const int64_t want = (args.cols + kThreads - 1) / kThreads, cap = (int64_t)sm_count() * 8;
-    wide_colsum_kernel<T><<<(unsigned)(want < cap ? want : cap), kThreads, 0, l.stream>>>(a, lda, (int)args.rows, args.cols, args.xr,
+    launch_chained(wide_colsum_kernel<T>, dim3((unsigned)(want < cap ? want : cap)), dim3(kThreads), 0, l.stream, a, lda, (int)args.rows, args.cols, args.xr,
                                                                                    incx, alpha, beta, args.y, incy);
     return check_launch();
   }
@@ -73,7 +73,7 @@ static int gemv_impl(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t
       args.ctiles_per_cta = 1;
       args.rows_per_cta = args.rows;
       args.direct = 0;
-      block_colsum_kernel<T><<<grid, kThreads, 0, l.stream>>>(a, args.rows, ppr, args.xr, incx, args.colpart, nsteps);
+      launch_chained(block_colsum_kernel<T>, dim3(grid), dim3(kThreads), 0, l.stream, a, args.rows, ppr, args.xr, incx, args.colpart, nsteps);
       if (int st = check_launch()) return st;
       launch_finalize<T, GemvCol, 32>(l, args, 1, (int)args.cols, args.cols);
       return check_launch();
@@ -93,7 +93,7 @@ static int gemv_impl(const b2_ctx* ctx, int order, int trans, int64_t m, int64_t
       args.ctiles_per_cta = 1;
       args.rows_per_cta = args.rows;
       args.direct = 0;
-      skinny_colsum_kernel<T><<<grid, kThreads, 0, l.stream>>>(a, args.rows, ppr, args.xr, incx, args.colpart, nsteps);
+      launch_chained(skinny_colsum_kernel<T>, dim3(grid), dim3(kThreads), 0, l.stream, a, args.rows, ppr, args.xr, incx, args.colpart, nsteps);
       if (int st = check_launch()) return st;
       launch_finalize<T, GemvCol, 32>(l, args, 1, (int)args.cols, args.cols);
       return check_launch();

@@ -11,6 +11,8 @@ __global__ void __launch_bounds__(kThreads) ger_kernel(T* __restrict__ a, int64_
                                                        const T* __restrict__ xr, int64_t incxr,
                                                        const T* __restrict__ yc, int64_t incyc, T alpha,
                                                        int64_t rows_per_cta, int nct) {
+  grid_dep_wait();
+  grid_dep_launch();
   constexpr int LPR = S::LPR, CU = S::CU, RU = S::RU, G = S::G, RB = S::RB;
   constexpr int TC = LPR * V * CU;
   using P = Pack<T, V>;
@@ -103,7 +105,7 @@ static int ger_launch(const Launch& l, T* a, int64_t lda, int64_t rows, int64_t 
   const int64_t rows_per_cta = (int64_t)S::RB * knob(kKnobGerRows);
   const int64_t nrs = (rows + rows_per_cta - 1) / rows_per_cta;
   if (nrs * nct > 0x7fffffff) return B2_STATUS_NOT_IMPLEMENTED;
-  ger_kernel<T, V, S><<<(unsigned)(nrs * nct), kThreads, 0, l.stream>>>(a, lda, rows, cols, xr, incxr, yc, incyc, alpha,
+  launch_chained(ger_kernel<T, V, S>, dim3((unsigned)(nrs * nct)), dim3(kThreads), 0, l.stream, a, lda, rows, cols, xr, incxr, yc, incyc, alpha,
                                                                         rows_per_cta, nct);
   return check_launch();
 }
@@ -149,7 +151,7 @@ static int ger_impl(const b2_ctx* ctx, int order, int64_t m, int64_t n, T alpha,
   // (measured: the element-wise walk wins in double; in float the pack kernels stay ahead)
   if (knob(kKnobNarrowBlock) && sizeof(T) == 8 && wide_applies<T>(rows, cols)) {
     const int64_t want = (cols + kThreads - 1) / kThreads, cap = (int64_t)sm_count() * 8;
-    wide_ger_kernel<T><<<(unsigned)(want < cap ? want : cap), kThreads, 0, l.stream>>>(a, lda, (int)rows, cols, xr, incxr, yc, incyc,
+    launch_chained(wide_ger_kernel<T>, dim3((unsigned)(want < cap ? want : cap)), dim3(kThreads), 0, l.stream, a, lda, (int)rows, cols, xr, incxr, yc, incyc,
                                                                                 alpha);
     return check_launch();
   }

@@ -74,6 +74,8 @@ struct RotmOp {
 template <typename T, class Op, int NV>
 __global__ void __launch_bounds__(kThreads) l1_map_unit(Op op, T* __restrict__ x, T* __restrict__ y, int64_t n,
                                                         int64_t head, int64_t nvec, int64_t nchunks) {
+  grid_dep_wait();
+  grid_dep_launch();
   constexpr int V = VecLen<T>::value;
   using P = Pack<T, V>;
   T* xv = x + head;
@@ -140,6 +142,8 @@ template <typename T, class Op, int NE>
 __global__ void __launch_bounds__(kThreads) l1_map_strided(Op op, T* __restrict__ x, int64_t incx,
                                                            T* __restrict__ y, int64_t incy, int64_t n,
                                                            int64_t nchunks) {
+  grid_dep_wait();
+  grid_dep_launch();
   for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
     const int64_t i0 = chunk * (int64_t)(kThreads * NE) + threadIdx.x;
     T a[NE], b[NE];
@@ -340,6 +344,8 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
                                                            int64_t head, int64_t nvec, int64_t nchunks,
                                                            typename Op::Acc* partials, unsigned* ticket,
                                                            typename Op::Out* result) {
+  grid_dep_wait();
+  grid_dep_launch();
   constexpr int V = VecLen<T>::value;
   using P = Pack<T, V>;
   using Acc = typename Op::Acc;
@@ -445,6 +451,8 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_strided(const T* __restric
                                                               const T* __restrict__ y, int64_t incy, int64_t n,
                                                               int64_t nchunks, typename Op::Acc* partials,
                                                               unsigned* ticket, typename Op::Out* result) {
+  grid_dep_wait();
+  grid_dep_launch();
   using Acc = typename Op::Acc;
   Acc r = Op::init();
   if constexpr (Op::kArgmax) {
@@ -500,6 +508,8 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_strided(const T* __restric
 
 // sdsdot's last step: result = (float)(sb + the double-accumulated dot), rounded once.
 __global__ void sdsdot_finish(const double* __restrict__ acc, float sb, float* __restrict__ result) {
+  grid_dep_wait();
+  grid_dep_launch();
   *result = (float)((double)sb + *acc);
 }
 
@@ -557,13 +567,12 @@ static int run_map(const b2_ctx* ctx, Op op, int64_t n, T* x, int64_t incx, T* y
     const int64_t nvec = (n - head) / V;
     const int64_t nchunks = (nvec + kThreads * NV - 1) / (kThreads * NV);
     const int64_t grid = nchunks < 1 ? 1 : (nchunks > (1 << 30) ? (1 << 30) : nchunks);
-    l1_map_unit<T, Op, NV><<<(unsigned)grid, kThreads, 0, l.stream>>>(op, x, two ? y : x, n, head, nvec, nchunks);
+    launch_chained(l1_map_unit<T, Op, NV>, dim3((unsigned)grid), dim3(kThreads), 0, l.stream, op, x, two ? y : x, n, head, nvec, nchunks);
   } else {
     constexpr int NE = 8;
     const int64_t nchunks = (n + kThreads * NE - 1) / (kThreads * NE);
     const int64_t grid = nchunks > (1 << 30) ? (1 << 30) : nchunks;
-    l1_map_strided<T, Op, NE><<<(unsigned)grid, kThreads, 0, l.stream>>>(
-        op, vec_base(x, n, incx), incx, two ? vec_base(y, n, incy) : x, two ? incy : 1, n, nchunks);
+    launch_chained(l1_map_strided<T, Op, NE>, dim3((unsigned)grid), dim3(kThreads), 0, l.stream, op, vec_base(x, n, incx), incx, two ? vec_base(y, n, incy) : x, two ? incy : 1, n, nchunks);
   }
   return check_launch();
 }
@@ -597,7 +606,7 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
     static WaveCache wc;
     const int wave = one_wave(l1_reduce_unit<T, Op, NV>, cap, wc);
     const int64_t grid = nchunks < 1 ? 1 : (nchunks > wave ? wave : nchunks);
-    l1_reduce_unit<T, Op, NV><<<(unsigned)grid, kThreads, 0, l.stream>>>(x, Op::RY ? y : x, n, head, nvec, nchunks,
+    launch_chained(l1_reduce_unit<T, Op, NV>, dim3((unsigned)grid), dim3(kThreads), 0, l.stream, x, Op::RY ? y : x, n, head, nvec, nchunks,
                                                                         partials, ticket, result);
   } else if (sizeof(T) == 4 && incx == 2 && (!Op::RY || incy == 2) && same_head<T>(x, y, Op::RY, &head)) {
     // (float only: for double, where a pack holds a single vector element, the strided kernel is the faster one)
@@ -609,7 +618,7 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
     static WaveCache wc;
     const int wave = one_wave(l1_reduce_unit<T, Op, NV, 2>, cap, wc);
     const int64_t grid = nchunks < 1 ? 1 : (nchunks > wave ? wave : nchunks);
-    l1_reduce_unit<T, Op, NV, 2><<<(unsigned)grid, kThreads, 0, l.stream>>>(x, Op::RY ? y : x, span, head, nvec, nchunks,
+    launch_chained(l1_reduce_unit<T, Op, NV, 2>, dim3((unsigned)grid), dim3(kThreads), 0, l.stream, x, Op::RY ? y : x, span, head, nvec, nchunks,
                                                                            partials, ticket, result);
   } else {
     constexpr int NE = Op::RY ? 8 : 16;
@@ -617,8 +626,7 @@ static int run_reduce(const b2_ctx* ctx, int64_t n, const T* x, int64_t incx, co
     static WaveCache wc;
     const int wave = one_wave(l1_reduce_strided<T, Op, NE>, cap, wc);
     const int64_t grid = nchunks > wave ? wave : nchunks;
-    l1_reduce_strided<T, Op, NE><<<(unsigned)grid, kThreads, 0, l.stream>>>(
-        vec_base(x, n, incx), incx, Op::RY ? vec_base(y, n, incy) : x, Op::RY ? incy : 1, n, nchunks, partials, ticket,
+    launch_chained(l1_reduce_strided<T, Op, NE>, dim3((unsigned)grid), dim3(kThreads), 0, l.stream, vec_base(x, n, incx), incx, Op::RY ? vec_base(y, n, incy) : x, Op::RY ? incy : 1, n, nchunks, partials, ticket,
         result);
   }
   return check_launch();
@@ -763,7 +771,7 @@ int b2_sdsdot(const b2_ctx* ctx, int64_t n, float sb, const float* x, int64_t in
   if (l.scratch_bytes < off + sizeof(double)) return B2_STATUS_WORKSPACE_TOO_SMALL;
   double* acc = reinterpret_cast<double*>(l.scratch + off);
   if (int st = run_reduce<float, DsdotOp>(ctx, n, x, incx, y, incy, acc)) return st;
-  sdsdot_finish<<<1, 1, 0, l.stream>>>(acc, sb, result);
+  launch_chained(sdsdot_finish, dim3(1), dim3(1), 0, l.stream, acc, sb, result);
   return check_launch();
 }
 

@@ -87,7 +87,8 @@ __global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args
   constexpr int TC = LPR * V * CU;
   constexpr int NCT = K::COLOUT ? S::NCT : 1;
   using P = Pack<T, V>;
-  grid_dep_launch();  // lets a dependent finalize launch be scheduled early (it waits for us)
+  grid_dep_wait();
+  grid_dep_launch();  // the next kernel of the stream (often this call's finalize pass) may be scheduled early
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane / LPR, q = lane % LPR;
@@ -313,6 +314,7 @@ __global__ void __launch_bounds__(kThreads) l2_finalize(const L2Args<T> p, int R
   constexpr int OUTB = kThreads / SLICES;
   __shared__ T sm[SLICES][OUTB];
   grid_dep_wait();
+  grid_dep_launch();
   const int o = threadIdx.x % OUTB, slice = threadIdx.x / OUTB;
   const int64_t nout = K::ROWOUT ? p.rows : p.cols;
   const int64_t i = (int64_t)blockIdx.x * OUTB + o;
@@ -354,6 +356,8 @@ __global__ void __launch_bounds__(kThreads) l2_finalize(const L2Args<T> p, int R
 // y <- beta*y (alpha == 0 shortcut); beta == 0 writes zeros without reading.
 template <typename T>
 __global__ void __launch_bounds__(kThreads) l2_scale_y(T* y, int64_t incy, int64_t n, T beta) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (i < n) y[i * incy] = beta == T(0) ? T(0) : beta * y[i * incy];
 }
@@ -420,7 +424,7 @@ static int l2_launch_shape(const Launch& l, L2Args<T> args, int64_t rows_per_cta
   }
   const int64_t nblocks = (int64_t)args.nrs * args.ncs;
   if (nblocks > 0x7fffffff) return B2_STATUS_NOT_IMPLEMENTED;
-  l2_tile_kernel<T, V, K, S><<<(unsigned)nblocks, kThreads, 0, l.stream>>>(args);
+  launch_chained(l2_tile_kernel<T, V, K, S>, dim3((unsigned)nblocks), dim3(kThreads), 0, l.stream, args);
   if (int st = check_launch()) return st;
   if (!args.direct) {
     const int64_t nout = K::ROWOUT ? args.rows : args.cols;
@@ -521,7 +525,7 @@ static L2Plan plan_colout(const L2Args<T>& a, bool narrow_ok, int64_t rows_per_c
 template <typename T>
 static int scale_y(const Launch& l, T* y, int64_t incy, int64_t n, T beta) {
   if (beta == T(1) || n == 0) return B2_STATUS_OK;
-  l2_scale_y<T><<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, l.stream>>>(vec_base(y, n, incy), incy, n, beta);
+  launch_chained(l2_scale_y<T>, dim3((unsigned)((n + kThreads - 1) / kThreads)), dim3(kThreads), 0, l.stream, vec_base(y, n, incy), incy, n, beta);
   return check_launch();
 }
 

@@ -48,6 +48,8 @@ __global__ void __launch_bounds__(kThreads, 3) skinny_rowdot_kernel(const T* __r
                                                                     const T* __restrict__ x, int64_t incx, T alpha,
                                                                     T beta, T* __restrict__ y, int64_t incy,
                                                                     int64_t nchunks) {
+  grid_dep_wait();
+  grid_dep_launch();
   constexpr int V = VecLen<T>::value;
   using P = Pack<T, V>;
   __shared__ __align__(16) T xs[kSkinnyMaxPpr * V];
@@ -108,6 +110,8 @@ __global__ void __launch_bounds__(kThreads, 3) skinny_ger_kernel(T* __restrict__
                                                                  const T* __restrict__ xr, int64_t incxr,
                                                                  const T* __restrict__ yc, int64_t incyc, T alpha,
                                                                  int64_t nchunks) {
+  grid_dep_wait();
+  grid_dep_launch();
   constexpr int V = VecLen<T>::value;
   using P = Pack<T, V>;
   __shared__ __align__(16) T ys[kSkinnyMaxPpr * V];
@@ -169,6 +173,7 @@ __global__ void __launch_bounds__(kThreads, 4) skinny_colsum_kernel(const T* __r
   constexpr int V = VecLen<T>::value;
   using P = Pack<T, V>;
   __shared__ T sm[kWarps][32 * V];
+  grid_dep_wait();
   grid_dep_launch();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = 32 / ppr;
@@ -241,6 +246,8 @@ __global__ void __launch_bounds__(kThreads, 3) block_rowdot_kernel(const T* __re
                                                                    const T* __restrict__ x, int64_t incx, T alpha,
                                                                    T beta, T* __restrict__ y, int64_t incy,
                                                                    int64_t nsteps) {
+  grid_dep_wait();
+  grid_dep_launch();
   constexpr int V = VecLen<T>::value, U = kBlockUnroll;
   using P = Pack<T, V>;
   extern __shared__ __align__(16) unsigned char block_smem[];
@@ -294,6 +301,7 @@ __global__ void __launch_bounds__(kThreads, 4) block_colsum_kernel(const T* __re
   constexpr int V = VecLen<T>::value, U = kBlockUnroll;
   using P = Pack<T, V>;
   __shared__ T sm[kThreads * V];
+  grid_dep_wait();
   grid_dep_launch();
   const int t = (int)threadIdx.x, K = kThreads / ppr, G = K * ppr;
   const bool active = t < G;
@@ -351,7 +359,7 @@ static int block_rowdot(const Launch& l, const T* a, int64_t rows, int64_t cols,
   const int64_t nsteps = (rows + (int64_t)K * kBlockUnroll - 1) / ((int64_t)K * kBlockUnroll);
   const int64_t cap = (int64_t)sm_count() * 3;
   const size_t smem = sizeof(T) * (size_t)kBlockUnroll * K * (ppr | 1);
-  block_rowdot_kernel<T><<<(unsigned)(nsteps < cap ? nsteps : cap), kThreads, smem, l.stream>>>(a, rows, ppr, x, incx, alpha,
+  launch_chained(block_rowdot_kernel<T>, dim3((unsigned)(nsteps < cap ? nsteps : cap)), dim3(kThreads), smem, l.stream, a, rows, ppr, x, incx, alpha,
                                                                                           beta, y, incy, nsteps);
   return check_launch();
 }
@@ -375,6 +383,8 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads) wide_colsum_kernel(const T* __restrict__ a, int64_t lda, int rows, int64_t cols,
                                                                const T* __restrict__ xr, int64_t incxr, T alpha, T beta,
                                                                T* __restrict__ y, int64_t incy) {
+  grid_dep_wait();
+  grid_dep_launch();
   __shared__ T xs[kWideMaxRows];
   if (threadIdx.x < rows) xs[threadIdx.x] = __ldg(xr + threadIdx.x * incxr);
   __syncthreads();
@@ -400,6 +410,8 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads) wide_ger_kernel(T* __restrict__ a, int64_t lda, int rows, int64_t cols,
                                                             const T* __restrict__ xr, int64_t incxr,
                                                             const T* __restrict__ yc, int64_t incyc, T alpha) {
+  grid_dep_wait();
+  grid_dep_launch();
   __shared__ T xs[kWideMaxRows];
   if (threadIdx.x < rows) xs[threadIdx.x] = alpha * __ldg(xr + threadIdx.x * incxr);
   __syncthreads();
@@ -430,7 +442,7 @@ static int skinny_rowdot(const Launch& l, const T* a, int64_t rows, int64_t cols
                          T beta, T* y, int64_t incy) {
   const int ppr = (int)(cols / VecLen<T>::value);
   const int64_t nchunks = (rows + 31) / 32;
-  skinny_rowdot_kernel<T><<<skinny_grid<T>(nchunks), kThreads, 0, l.stream>>>(a, rows, ppr, x, incx, alpha, beta, y,
+  launch_chained(skinny_rowdot_kernel<T>, dim3(skinny_grid<T>(nchunks)), dim3(kThreads), 0, l.stream, a, rows, ppr, x, incx, alpha, beta, y,
                                                                              incy, nchunks);
   return check_launch();
 }
@@ -440,7 +452,7 @@ static int skinny_ger(const Launch& l, T* a, int64_t rows, int64_t cols, const T
                       int64_t incyc, T alpha) {
   const int ppr = (int)(cols / VecLen<T>::value);
   const int64_t nchunks = (rows + 31) / 32;
-  skinny_ger_kernel<T><<<skinny_grid<T>(nchunks), kThreads, 0, l.stream>>>(a, rows, ppr, xr, incxr, yc, incyc, alpha,
+  launch_chained(skinny_ger_kernel<T>, dim3(skinny_grid<T>(nchunks)), dim3(kThreads), 0, l.stream, a, rows, ppr, xr, incxr, yc, incyc, alpha,
                                                                           nchunks);
   return check_launch();
 }

@@ -56,6 +56,8 @@ __global__ void __launch_bounds__(kThreads, TWO ? 3 : 4) syr_kernel(T* __restric
                                                        const T* __restrict__ x, int64_t incx,
                                                        const T* __restrict__ y, int64_t incy, T alpha, bool lower,
                                                        int nct) {
+  grid_dep_wait();
+  grid_dep_launch();
   constexpr int kSyrCU = SyrShape<T, TWO>::CU, kSyrRU = SyrShape<T, TWO>::RU;
   constexpr int kSyrRows = kWarps * kSyrRU;  // rows per block
   constexpr int TC = 32 * V * kSyrCU;        // columns per block
@@ -169,7 +171,7 @@ static int syr_launch(const Launch& l, T* a, int64_t lda, int64_t n, const T* x,
   const int64_t nct = (n + TC - 1) / TC;
   const int64_t blocks = M * (nct * (nct + 1) / 2);
   if (blocks > 0x7fffffff) return B2_STATUS_NOT_IMPLEMENTED;
-  syr_kernel<T, V, TWO><<<(unsigned)blocks, kThreads, 0, l.stream>>>(a, lda, n, x, incx, y, incy, alpha, lower,
+  launch_chained(syr_kernel<T, V, TWO>, dim3((unsigned)blocks), dim3(kThreads), 0, l.stream, a, lda, n, x, incx, y, incy, alpha, lower,
                                                                      (int)nct);
   return check_launch();
 }

@@ -121,6 +121,7 @@ __global__ void __launch_bounds__(kThreads, 1) tri_tile_kernel(const TileArgs<T,
   constexpr bool WALK_ROWS = ROW;  // column-sum-only kinds walk down a block column
   constexpr int XCU = WALK_ROWS ? kUnitMax * TC : TC;  // most column values a unit needs
   using P = Pack<T, V>;
+  grid_dep_wait();
   grid_dep_launch();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* ring = reinterpret_cast<uint4*>(smem_raw);             // [kRing][TP][kThreads] packs
@@ -361,6 +362,7 @@ __global__ void __launch_bounds__(fin_warps<T>() * 32) tri_tile_finalize(const T
   constexpr bool WALK_ROWS = ROW;
   __shared__ T part[kFinWarps][33];
   grid_dep_wait();
+  grid_dep_launch();
   const int w = (int)(threadIdx.x >> 5), lane = (int)(threadIdx.x & 31);
   const int64_t i = (int64_t)blockIdx.x * 32 + lane;
   T s = T(0);
@@ -464,7 +466,7 @@ static int tri_tile_run_cap(const Launch& l, const T* a, int64_t lda, int64_t n,
   *handled = true;
   const int nunits = args.prefix[nmajor];
   const int grid = nunits < sm_count() ? nunits : sm_count();
-  kern<<<grid, kThreads, smem, l.stream>>>(args);
+  launch_chained(kern, dim3(grid), dim3(kThreads), smem, l.stream, args);
   if (int st = check_launch()) return st;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)((n + 31) / 32));

@@ -138,6 +138,8 @@ __device__ __forceinline__ double decode(const unsigned long long* w, double) {
 // NB^2 per unknown, and a 128 x 128 double block with its inverse would not fit in shared memory).
 template <typename T, int NB, int V, bool COLTYPE, bool BACKWARD, bool UNIT>
 __global__ void __launch_bounds__(kTT) trsv_kernel(const TrsvArgs<T> p) {
+  grid_dep_wait();
+  grid_dep_launch();
   // A tile is NB own unknowns x 64 source unknowns; in memory it is NB rows x 64 columns
   // (rows of op(A) contiguous) or 64 rows x NB columns (COLTYPE).
   constexpr int WS = NB + 8;        // row stride of W (16-byte row starts, conflict-free packs)
@@ -534,7 +536,7 @@ static int trsv_launch_one(const Launch& l, const TrsvArgs<T>& args) {
     (void)cudaGetLastError();
     return B2_STATUS_LAUNCH_FAILED;
   }
-  kern<<<args.nb, kTT, smem, l.stream>>>(args);
+  launch_chained(kern, dim3(args.nb), dim3(kTT), smem, l.stream, args);
   return check_launch();
 }
 

@@ -216,6 +216,8 @@ __device__ __forceinline__ void st4(double* p, double a, double b, double c, dou
 // L2 and the polling of global memory.
 template <typename T, bool COLTYPE, bool BACKWARD, bool UNIT, int CS>
 __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p) {
+  grid_dep_wait();
+  grid_dep_launch();
   constexpr int NB = Geo<T>::NB, V = Geo<T>::V, WPE = Words<T>::N;
   constexpr int RS = NB / 16;  // sub-block edge: 8 (float) / 4 (double)
   constexpr int E = RS * RS;
@@ -270,9 +272,6 @@ __global__ void __launch_bounds__(kT, 1) trsv_front_kernel(const FrontArgs<T> p)
     if (rank == 0u && ct == 0) {
       unsigned kk = 0xffffffffu;
       if (!wt.dead && ld_flag(wt.abort_word) == 0u) kk = atomicAdd(p.ctl + kCtlTrsvTicket, 1u);
-      // abort word up (raised in this call, or left by an earlier timed-out call on a workspace
-      // that was not reset): nothing more is solved, and the caller must be able to see that
-      else if (p.device_status) atomicExch(p.device_status, (int)B2_STATUS_TIMEOUT);
       // abort word up (raised in this call, or left by an earlier timed-out call on a workspace
       // that was not reset): nothing more is solved, and the caller must be able to see that
       else if (p.device_status) atomicExch(p.device_status, (int)B2_STATUS_TIMEOUT);
@@ -802,7 +801,7 @@ static int launch_one(const Launch& l, const FrontArgs<T>& args, int nb, bool wa
     return B2_STATUS_LAUNCH_FAILED;
   }
   const int grid = nb < sm_count() ? nb : sm_count();
-  kern<<<grid, kT, smem, l.stream>>>(args);
+  launch_chained(kern, dim3(grid), dim3(kT), smem, l.stream, args);
   return check_launch();
 }
 
