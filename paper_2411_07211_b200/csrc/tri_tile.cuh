@@ -27,10 +27,20 @@ namespace tt {
 // (measured: wider, flatter tiles -- 64 x 256 or 32 x 512 floats -- are slower here, they waste
 // more of the tiles that the diagonal cuts and make the units coarser)
 constexpr int kRing = 3;       // tiles (64 KB each) in the shared-memory ring
-constexpr int kNR = 8;         // rows of a tile a thread holds
+#ifndef B2_TT_NR
+#define B2_TT_NR 8
+#endif
+#ifndef B2_TT_UNITMAX
+#define B2_TT_UNITMAX 4
+#endif
+#ifndef B2_TT_BPS
+#define B2_TT_BPS 1
+#endif
+constexpr int kBlocksPerSm = B2_TT_BPS;
+constexpr int kNR = B2_TT_NR;  // rows of a tile a thread holds
 constexpr int kNP = 2;         // packs of each row a thread holds (16 lanes side by side, kNP groups of them)
 constexpr int kTR = 16 * kNR;  // tile rows
-constexpr int kUnitMax = 4;    // tiles per unit at most (1, 2 or 4)
+constexpr int kUnitMax = B2_TT_UNITMAX;  // tiles per unit at most (1, 2 or 4)
 constexpr int kMaxMajor = 2048;  // block rows (or column tiles) the unit table can hold
 
 // Elements of the queue of x values: one slot per unit that can be in flight.  The producer runs
@@ -116,7 +126,7 @@ __device__ __forceinline__ void cp_async_wait() {
 // multiplied.  Edge tiles use the same copies with a byte count that zero-fills what lies outside
 // the matrix.  The x values of a unit travel the same way.
 template <typename T, int CAP, bool ROW, bool COL, int TRI, bool UNIT, bool SYM>
-__global__ void __launch_bounds__(kThreads, 1) tri_tile_kernel(const TileArgs<T, CAP> p) {
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm) tri_tile_kernel(const TileArgs<T, CAP> p) {
   constexpr int V = VecLen<T>::value, TC = 16 * kNP * V, NR = kNR, HR = NR / 2, NP = kNP, TP = NR * NP;
   constexpr bool WALK_ROWS = ROW;  // column-sum-only kinds walk down a block column
   constexpr int XCU = WALK_ROWS ? kUnitMax * TC : TC;  // most column values a unit needs
@@ -431,12 +441,14 @@ static int tri_tile_run_cap(const Launch& l, const T* a, int64_t lda, int64_t n,
   args.incx = incx;
   args.nbr = (int)nbr;
   args.nct = (int)nct;
-  // a few thousand units keep the tail short; beyond that, longer units mean fewer partials
+  // longer units mean fewer partials, fewer reductions and fewer block-wide barriers per tile; a
+  // dozen units per block keep the tail short (measured at 4096 tiles on 148 blocks: units of 2
+  // take symv from 57 / 53 us (upper / lower, float) to 50.5 us, units of 4 to 52 / 50 us)
   const int64_t tiles = nbr * nct / 2;
-  const int64_t want = tiles / ((int64_t)sm_count() * 16);
-  args.unit = (want >= 4 && kUnitMax >= 4) ? 4 : (want >= 2 && kUnitMax >= 2) ? 2 : 1;
+  const int64_t per_block = tiles / sm_count();
+  args.unit = (per_block >= 48 && kUnitMax >= 4) ? 4 : (per_block >= 12 && kUnitMax >= 2) ? 2 : 1;
   const int64_t forced = knob(kKnobTriTileUnit);
-  if (forced == 1 || forced == 2 || forced == 4) args.unit = (int)forced;
+  if ((forced == 1 || forced == 2 || forced == 4) && forced <= kUnitMax) args.unit = (int)forced;
   const int nmajor = WALK_ROWS ? args.nbr : args.nct;
   int ngroups = 0;
   for (int i = 0; i < nmajor; ++i) {
@@ -465,7 +477,7 @@ static int tri_tile_run_cap(const Launch& l, const T* a, int64_t lda, int64_t n,
   }
   *handled = true;
   const int nunits = args.prefix[nmajor];
-  const int grid = nunits < sm_count() ? nunits : sm_count();
+  const int grid = nunits < sm_count() * kBlocksPerSm ? nunits : sm_count() * kBlocksPerSm;
   launch_chained(kern, dim3(grid), dim3(kThreads), smem, l.stream, args);
   if (int st = check_launch()) return st;
   cudaLaunchConfig_t cfg = {};
