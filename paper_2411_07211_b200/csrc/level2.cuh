@@ -223,39 +223,55 @@ __global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args
             }
       } else {
         // Diagonal tiles and column edges inside a pack: local 32-bit indices; d = (first column)
-        // - (first row), so element (li, lj) lies on the diagonal when d + lj == li.
+        // - (first row), so element (li, lj) lies on the diagonal when d + lj == li.  All loads
+        // of the tile go out together, each under its own predicate (a pack wholly outside the
+        // triangle or the matrix is not read), and only then are the elements masked: loads
+        // issued one by one between the branches made such a tile last several memory latencies.
         const int64_t d64 = c0 - rb;
         const int d = (int)(d64 > (1 << 24) ? (1 << 24) : d64 < -(1 << 24) ? -(1 << 24) : d64);
         const int nc = (int)(c1 - c0);
         const T* at = a_rb + c0;
+        P av[RU][CU];
 #pragma unroll
         for (int ru = 0; ru < RU; ++ru) {
           const int li = lrow0 + ru * kWarps * G;
-          if (li >= nr) continue;
 #pragma unroll
           for (int u = 0; u < CU; ++u) {
             const int lc = (u * LPR + q) * V;
-            if (lc >= nc) continue;
-            if (K::TRI == TRI_UPPER && d + lc + V - 1 < li) continue;  // pack wholly outside
-            if (K::TRI == TRI_LOWER && d + lc > li) continue;
-            const T* ap = at + ru * rstride + u * (LPR * V);
-            P av;
-            if (V > 1 && lc + V <= nc) {
-              av = ld_nc<T, V>(ap);
-            } else {
+            bool use = li < nr && lc < nc;
+            if (K::TRI == TRI_UPPER) use = use && d + lc + V - 1 >= li;
+            if (K::TRI == TRI_LOWER) use = use && d + lc <= li;
 #pragma unroll
-              for (int e = 0; e < V; ++e) av.v[e] = (lc + e < nc) ? __ldg(ap + e) : T(0);
+            for (int e = 0; e < V; ++e) av[ru][u].v[e] = T(0);
+            const T* ap = at + ru * rstride + u * (LPR * V);
+            if (use) {
+              if (V == 1 || lc + V <= nc) {
+                av[ru][u] = ld_nc<T, V>(ap);
+              } else {
+#pragma unroll
+                for (int e = 0; e < V; ++e)
+                  if (lc + e < nc) av[ru][u].v[e] = __ldg(ap + e);
+              }
             }
+          }
+        }
+#pragma unroll
+        for (int ru = 0; ru < RU; ++ru) {
+          const int li = lrow0 + ru * kWarps * G;
+#pragma unroll
+          for (int u = 0; u < CU; ++u) {
+            const int lc = (u * LPR + q) * V;
 #pragma unroll
             for (int e = 0; e < V; ++e) {
               const int lj = lc + e;
-              if (lj >= nc) continue;
-              if (K::TRI == TRI_UPPER && d + lj < li) continue;
-              if (K::TRI == TRI_LOWER && d + lj > li) continue;
+              bool in = li < nr && lj < nc;
+              if (K::TRI == TRI_UPPER) in = in && d + lj >= li;
+              if (K::TRI == TRI_LOWER) in = in && d + lj <= li;
               const bool dg = (K::TRI != TRI_FULL) && (d + lj == li);
-              const T v = (K::UNIT && dg) ? T(1) : av.v[e];
-              if (K::ROWOUT) rowacc[ru] = v * xcv[c][u][e] + rowacc[ru];
-              if (K::COLOUT && !(K::SYM && dg)) colacc[c][u][e] = v * xrv[ru] + colacc[c][u][e];
+              const T v = (K::UNIT && dg) ? T(1) : av[ru][u].v[e];
+              // (a select, not a product with zero: x may hold infinities where the triangle ends)
+              if (K::ROWOUT) rowacc[ru] = in ? v * xcv[c][u][e] + rowacc[ru] : rowacc[ru];
+              if (K::COLOUT && !(K::SYM && dg)) colacc[c][u][e] = in ? v * xrv[ru] + colacc[c][u][e] : colacc[c][u][e];
             }
           }
         }
