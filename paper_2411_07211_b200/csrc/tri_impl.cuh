@@ -61,7 +61,12 @@ static int symv_impl(const b2_ctx* ctx, int order, int uplo, int64_t n, T alpha,
   args.incy = incy;
   // the stored triangle as it sits in the row-major view of the buffer
   const bool upper = (order == B2_ROW_MAJOR) == (uplo == B2_UPPER);
-  if (knob(kKnobTriTile)) {  // 16-byte aligned matrices: the tile kernel with the shared-memory ring
+  // The tile kernel with the shared-memory ring (16-byte aligned matrices) is the faster one while
+  // the triangle is small (n = 4096: 13 us against 19 us in float); from about 64 MiB of triangle
+  // on the general tile kernel streams faster (n = 32768 float: 320 us against 357 us).  Knob value
+  // 2 forces the ring kernel at every size (tests).
+  const bool small = (double)n * (double)n * sizeof(T) / 2 <= 64.0 * 1024 * 1024;
+  if (knob(kKnobTriTile) == 2 || (knob(kKnobTriTile) == 1 && small)) {
     bool handled = false;
     const int st = upper ? tt::tri_tile_run<T, true, true, TRI_UPPER, false, true>(l, a, lda, n, args.xc, incx, alpha, beta,
                                                                                   args.y, incy, &handled)

@@ -126,11 +126,20 @@ TRI_SIZES = [1, 2, 5, 31, 64, 65, 127, 128, 129, 200, 513, 1100]
 TRI_CASES = [(0, 0, 1), (1, 0, 2), (4, 1, -1), (0, 0, 2)]  # pad, offset, inc
 
 
+@pytest.fixture(params=[0, 2], ids=["general-kernel", "ring-kernel"])
+def symv_kernel(request, b2):
+    """symv picks its kernel by the size of the triangle; both are run on every test size."""
+    old = b2.get_tuning(b2.KNOB_TRI_TILE)
+    b2.set_tuning(b2.KNOB_TRI_TILE, request.param)
+    yield request.param
+    b2.set_tuning(b2.KNOB_TRI_TILE, old)
+
+
 @pytest.mark.parametrize("dtype", DTYPES)
 @pytest.mark.parametrize("order", ORDERS)
 @pytest.mark.parametrize("uplo", UPLOS)
 @pytest.mark.parametrize("n", TRI_SIZES)
-def test_symv(b2, ctx, dtype, order, uplo, n):
+def test_symv(b2, ctx, dtype, order, uplo, n, symv_kernel):
     for (pad, offset, inc), beta in zip(TRI_CASES, [0.5, 0.0, 0.5, 0.0]):
         lda = n + pad
         a = tri_buf(9, n, lda, dtype, order, uplo, orc.NON_UNIT)

@@ -118,14 +118,22 @@ def test_triangular_config_sizes(b2, ctx, dtype, n):
     rows = sample(n, n)
     tidx = torch.from_numpy(rows).cuda()
     for uplo in (orc.UPPER, orc.LOWER):
-        y = dvec(seed, 8, n, dtype)
-        b2.symv(ctx, orc.ROW_MAJOR, uplo, n, 1.25, a, n, dvec(seed, 7, n, dtype), 1, 0.5, y, 1)
-        got = y[tidx].cpu().numpy()
-        for i, g in zip(rows, got):
+        gots = []
+        for kernel in (0, 2):  # the general tile kernel, then the one with the shared-memory ring
+            old = b2.get_tuning(b2.KNOB_TRI_TILE)
+            b2.set_tuning(b2.KNOB_TRI_TILE, kernel)
+            try:
+                y = dvec(seed, 8, n, dtype)
+                b2.symv(ctx, orc.ROW_MAJOR, uplo, n, 1.25, a, n, dvec(seed, 7, n, dtype), 1, 0.5, y, 1)
+                gots.append(y[tidx].cpu().numpy())
+            finally:
+                b2.set_tuning(b2.KNOB_TRI_TILE, old)
+        for k, i in enumerate(rows):
             row = op_row(seed, stream, n, dtype, uplo, orc.NO_TRANS, orc.NON_UNIT, i, symmetric=True)
             out = hy[i:i + 1].copy()
             absterms = orc.gemv(orc.ROW_MAJOR, orc.NO_TRANS, 1, n, dtype(1.25), row, n, hx, 1, dtype(0.5), out, 1)
-            assert_close(g, out[0], absterms[0], dtype, f"symv uplo {uplo} row {i}")
+            for kernel, got in zip(("general", "ring"), gots):
+                assert_close(got[k], out[0], absterms[0], dtype, f"symv ({kernel} kernel) uplo {uplo} row {i}")
         for trans in (orc.NO_TRANS, orc.TRANS):
             for diag in (orc.NON_UNIT, orc.UNIT):
                 x = dvec(seed, 7, n, dtype)
