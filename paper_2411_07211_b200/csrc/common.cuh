@@ -137,6 +137,29 @@ __device__ __forceinline__ Pack<T, N> ld_nc(const T* p) {
   return r;
 }
 
+// The same load under a predicate, zeros otherwise, as ONE instruction sequence without a branch.
+// (`if (c) v = ld_nc(p)` compiles to a branch around the load and a copy of the loaded registers
+// where the paths meet; the copy waits for the load, so several such loads in a row go out one
+// memory latency after the other.)
+template <typename T, int N>
+__device__ __forceinline__ Pack<T, N> ld_nc_if(const T* p, bool pred) {
+  Pack<T, N> r = {};
+  if (pred && !B2_GUARD(p, sizeof(T) * N)) pred = false;
+  if constexpr (sizeof(T) * N == 16) {
+    uint4 t;
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %5, 0;\n\tmov.u32 %0, 0;\n\tmov.u32 %1, 0;\n\tmov.u32 %2, 0;\n\tmov.u32 %3, 0;\n\t"
+        "@q ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
+        : "=&r"(t.x), "=&r"(t.y), "=&r"(t.z), "=&r"(t.w)
+        : "l"(p), "r"((unsigned)pred));
+    r = *reinterpret_cast<Pack<T, N>*>(&t);
+  } else {
+    static_assert(N == 1, "packs are 16 bytes or one element");
+    r.v[0] = pred ? __ldg(p) : T(0);
+  }
+  return r;
+}
+
 // Read-only load of reused data (the x vectors): cached in L1.
 template <typename T, int N>
 __device__ __forceinline__ Pack<T, N> ld_ro(const T* p) {

@@ -92,8 +92,14 @@ __global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane / LPR, q = lane % LPR;
-  const int cs = blockIdx.x % p.ncs;
-  const int64_t rs = blockIdx.x / p.ncs;
+  // Blocks start in index order.  In an upper triangle the bottom-right blocks are the ones that the
+  // matrix edge cuts (the last column tile, ragged when n is not a multiple of the tile, is there the
+  // LONGEST column); started last and running alone they would be the tail (measured in double at
+  // n = 8190, column sums: 74 us against 48), so the order is reversed and the last block to start
+  // is the small one in the top-left corner.
+  const unsigned bidx = K::TRI == TRI_UPPER ? gridDim.x - 1u - blockIdx.x : blockIdx.x;
+  const int cs = (int)(bidx % (unsigned)p.ncs);
+  const int64_t rs = bidx / (unsigned)p.ncs;
   const int64_t r_begin = rs * p.rows_per_cta;
   const int64_t r_end = min(p.rows, r_begin + p.rows_per_cta);
   const int ct_begin = cs * p.ctiles_per_cta;
@@ -207,9 +213,7 @@ __global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args
           const bool rok = lrow0 + ru * kWarps * G < nr;
 #pragma unroll
           for (int u = 0; u < CU; ++u) {
-#pragma unroll
-            for (int e = 0; e < V; ++e) av[ru][u].v[e] = T(0);
-            if (rok && u * LPR + q < npk) av[ru][u] = ld_nc<T, V>(at + ru * rstride + u * (LPR * V));
+            av[ru][u] = ld_nc_if<T, V>(at + ru * rstride + u * (LPR * V), rok && u * LPR + q < npk);
           }
         }
 #pragma unroll
@@ -241,17 +245,23 @@ __global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args
             bool use = li < nr && lc < nc;
             if (K::TRI == TRI_UPPER) use = use && d + lc + V - 1 >= li;
             if (K::TRI == TRI_LOWER) use = use && d + lc <= li;
+            av[ru][u] = ld_nc_if<T, V>(at + ru * rstride + u * (LPR * V), use && (V == 1 || lc + V <= nc));
+          }
+        }
+        if (V > 1 && nc % V != 0) {  // the rows end inside a pack: that pack element by element
 #pragma unroll
-            for (int e = 0; e < V; ++e) av[ru][u].v[e] = T(0);
-            const T* ap = at + ru * rstride + u * (LPR * V);
-            if (use) {
-              if (V == 1 || lc + V <= nc) {
-                av[ru][u] = ld_nc<T, V>(ap);
-              } else {
+          for (int ru = 0; ru < RU; ++ru) {
+            const int li = lrow0 + ru * kWarps * G;
 #pragma unroll
-                for (int e = 0; e < V; ++e)
-                  if (lc + e < nc) av[ru][u].v[e] = __ldg(ap + e);
-              }
+            for (int u = 0; u < CU; ++u) {
+              const int lc = (u * LPR + q) * V;
+              bool use = li < nr && lc < nc && lc + V > nc;
+              if (K::TRI == TRI_UPPER) use = use && d + lc + V - 1 >= li;
+              if (K::TRI == TRI_LOWER) use = use && d + lc <= li;
+              const T* ap = at + ru * rstride + u * (LPR * V);
+#pragma unroll
+              for (int e = 0; e < V; ++e)
+                if (use && lc + e < nc) av[ru][u].v[e] = __ldg(ap + e);
             }
           }
         }
@@ -341,18 +351,40 @@ __global__ void __launch_bounds__(kThreads) l2_finalize(const L2Args<T> p, int R
       const int64_t r_end = min(p.rows, (rs + 1) * p.rows_per_cta);
       const int64_t rb = (i / RB) * RB;  // rows_per_cta is a multiple of RB
       const int64_t rb_end = min(rb + RB, r_end);
-      for (int cs = slice; cs < p.ncs; cs += SLICES) {
-        const int64_t c_lo = (int64_t)cs * p.ctiles_per_cta * TC;
-        const int64_t c_hi = min(p.cols, c_lo + (int64_t)p.ctiles_per_cta * TC);
-        if (region_active<K::TRI>(rb, rb_end, c_lo, c_hi)) s += __ldcg(p.rowpart + (int64_t)cs * p.rows + i);
+      // four partials per trip, their loads issued together (a load behind each test would
+      // cost one L2 round trip per partial); added in the same order as one by one
+      for (int cs0 = slice; cs0 < p.ncs; cs0 += 4 * SLICES) {
+        T v[4];
+        bool act[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int cs = cs0 + k * SLICES;
+          const int64_t c_lo = (int64_t)cs * p.ctiles_per_cta * TC;
+          const int64_t c_hi = min(p.cols, c_lo + (int64_t)p.ctiles_per_cta * TC);
+          act[k] = cs < p.ncs && region_active<K::TRI>(rb, rb_end, c_lo, c_hi);
+          v[k] = act[k] ? __ldcg(p.rowpart + (int64_t)cs * p.rows + i) : T(0);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (act[k]) s += v[k];
       }
     }
     if (K::COLOUT) {
       const int64_t span = (int64_t)TC * p.ctiles_per_cta;  // columns of one block
       const int64_t c_lo = (i / span) * span, c_hi = min(p.cols, c_lo + span);
-      for (int64_t rs = slice; rs < p.nrs; rs += SLICES) {
-        const int64_t r_begin = rs * p.rows_per_cta, r_end = min(p.rows, r_begin + p.rows_per_cta);
-        if (region_active<K::TRI>(r_begin, r_end, c_lo, c_hi)) s += __ldcg(p.colpart + rs * p.cols + i);
+      for (int64_t rs0 = slice; rs0 < p.nrs; rs0 += 4 * SLICES) {
+        T v[4];
+        bool act[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int64_t rs = rs0 + k * SLICES;
+          const int64_t r_begin = rs * p.rows_per_cta, r_end = min(p.rows, r_begin + p.rows_per_cta);
+          act[k] = rs < p.nrs && region_active<K::TRI>(r_begin, r_end, c_lo, c_hi);
+          v[k] = act[k] ? __ldcg(p.colpart + rs * p.cols + i) : T(0);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (act[k]) s += v[k];
       }
     }
   }
