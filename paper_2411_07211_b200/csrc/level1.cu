@@ -364,7 +364,7 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
 #pragma unroll
       for (int k = 0; k < NV; ++k) {
         const int64_t v = v0 + (int64_t)k * kThreads;
-        if (v < nvec) px[k] = ld_nc<T, V>(xv + v * V);
+        px[k] = ld_nc_if<T, V>(xv + v * V, v < nvec);
       }
 #pragma unroll
       for (int k = 0; k < NV; ++k) {

@@ -71,7 +71,7 @@ __global__ void __launch_bounds__(kThreads, 3) skinny_rowdot_kernel(const T* __r
 #pragma unroll
       for (int g = 0; g < kSkinnyGroup; ++g) {
         const int pos = (k0 + g) * 32 + lane;
-        if (k0 + g < ppr && pos < npacks) av[g] = ld_nc<T, V>(reinterpret_cast<const T*>(src + pos));
+        av[g] = ld_nc_if<T, V>(reinterpret_cast<const T*>(src + pos), k0 + g < ppr && pos < npacks);
       }
 #pragma unroll
       for (int g = 0; g < kSkinnyGroup; ++g) {
@@ -192,13 +192,8 @@ __global__ void __launch_bounds__(kThreads, 4) skinny_colsum_kernel(const T* __r
     for (int k = 0; k < kColsumGroup; ++k) {
       const int64_t row = row0 + k * G + g;
       const bool ok = active && row < rows;
-      xv[k] = T(0);
-#pragma unroll
-      for (int e = 0; e < V; ++e) av[k].v[e] = T(0);
-      if (ok) {
-        av[k] = ld_nc<T, V>(reinterpret_cast<const T*>(src + (int64_t)k * G * ppr));
-        xv[k] = __ldg(xr + row * incxr);
-      }
+      av[k] = ld_nc_if<T, V>(reinterpret_cast<const T*>(src + (int64_t)k * G * ppr), ok);
+      xv[k] = ok ? __ldg(xr + row * incxr) : T(0);
     }
 #pragma unroll
     for (int k = 0; k < kColsumGroup; ++k)
@@ -265,9 +260,7 @@ __global__ void __launch_bounds__(kThreads, 3) block_rowdot_kernel(const T* __re
     P av[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-#pragma unroll
-      for (int e = 0; e < V; ++e) av[u].v[e] = T(0);
-      if (active && row0 + u * K + r < rows) av[u] = ld_nc<T, V>(reinterpret_cast<const T*>(src + (int64_t)u * G));
+      av[u] = ld_nc_if<T, V>(reinterpret_cast<const T*>(src + (int64_t)u * G), active && row0 + u * K + r < rows);
     }
     if (active) {
 #pragma unroll
@@ -318,13 +311,8 @@ __global__ void __launch_bounds__(kThreads, 4) block_colsum_kernel(const T* __re
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int64_t row = row0 + u * K + r;
-      xv[u] = T(0);
-#pragma unroll
-      for (int e = 0; e < V; ++e) av[u].v[e] = T(0);
-      if (active && row < rows) {
-        av[u] = ld_nc<T, V>(reinterpret_cast<const T*>(src + (int64_t)u * G));
-        xv[u] = __ldg(xr + row * incxr);
-      }
+      av[u] = ld_nc_if<T, V>(reinterpret_cast<const T*>(src + (int64_t)u * G), active && row < rows);
+      xv[u] = (active && row < rows) ? __ldg(xr + row * incxr) : T(0);
     }
 #pragma unroll
     for (int u = 0; u < U; ++u)
