@@ -213,7 +213,9 @@ __global__ void __launch_bounds__(kThreads, S::MINB) l2_tile_kernel(const L2Args
           const bool rok = lrow0 + ru * kWarps * G < nr;
 #pragma unroll
           for (int u = 0; u < CU; ++u) {
-            av[ru][u] = ld_nc_if<T, V>(at + ru * rstride + u * (LPR * V), rok && u * LPR + q < npk);
+#pragma unroll
+            for (int e = 0; e < V; ++e) av[ru][u].v[e] = T(0);
+            if (rok && u * LPR + q < npk) av[ru][u] = ld_nc<T, V>(at + ru * rstride + u * (LPR * V));
           }
         }
 #pragma unroll
@@ -353,6 +355,9 @@ __global__ void __launch_bounds__(kThreads) l2_finalize(const L2Args<T> p, int R
       const int64_t rb_end = min(rb + RB, r_end);
       // four partials per trip, their loads issued together (a load behind each test would
       // cost one L2 round trip per partial); added in the same order as one by one
+      if constexpr (K::TRI == TRI_FULL) {  // every partial exists: a plain loop, which the compiler pipelines
+        for (int cs = slice; cs < p.ncs; cs += SLICES) s += __ldcg(p.rowpart + (int64_t)cs * p.rows + i);
+      } else
       for (int cs0 = slice; cs0 < p.ncs; cs0 += 4 * SLICES) {
         T v[4];
         bool act[4];
@@ -372,6 +377,9 @@ __global__ void __launch_bounds__(kThreads) l2_finalize(const L2Args<T> p, int R
     if (K::COLOUT) {
       const int64_t span = (int64_t)TC * p.ctiles_per_cta;  // columns of one block
       const int64_t c_lo = (i / span) * span, c_hi = min(p.cols, c_lo + span);
+      if constexpr (K::TRI == TRI_FULL) {
+        for (int64_t rs = slice; rs < p.nrs; rs += SLICES) s += __ldcg(p.colpart + rs * p.cols + i);
+      } else
       for (int64_t rs0 = slice; rs0 < p.nrs; rs0 += 4 * SLICES) {
         T v[4];
         bool act[4];

@@ -260,7 +260,15 @@ __global__ void __launch_bounds__(kThreads, 3) block_rowdot_kernel(const T* __re
     P av[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      av[u] = ld_nc_if<T, V>(reinterpret_cast<const T*>(src + (int64_t)u * G), active && row0 + u * K + r < rows);
+      // (double: the branch-free load, 0.82 -> 0.92 of the copy rate at 40 columns; float measured
+      // 5 % faster with the branch, which the compiler there turns into a predicate itself)
+      if constexpr (sizeof(T) == 8) {
+        av[u] = ld_nc_if<T, V>(reinterpret_cast<const T*>(src + (int64_t)u * G), active && row0 + u * K + r < rows);
+      } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e) av[u].v[e] = T(0);
+        if (active && row0 + u * K + r < rows) av[u] = ld_nc<T, V>(reinterpret_cast<const T*>(src + (int64_t)u * G));
+      }
     }
     if (active) {
 #pragma unroll
