@@ -65,8 +65,11 @@ static int symv_impl(const b2_ctx* ctx, int order, int uplo, int64_t n, T alpha,
   // the triangle is small (n = 4096: 13 us against 19 us in float); from about 64 MiB of triangle
   // on the general tile kernel streams faster (n = 32768 float: 320 us against 357 us).  Knob value
   // 2 forces the ring kernel at every size (tests).
+  // (double, upper triangle: that kind of the general kernel spills 132 bytes per thread at its
+  // 64 registers and streams 10-15 % slower than the ring kernel at every size -- n = 32768:
+  // 780 us against 684 us)
   const bool small = (double)n * (double)n * sizeof(T) / 2 <= 64.0 * 1024 * 1024;
-  if (knob(kKnobTriTile) == 2 || (knob(kKnobTriTile) == 1 && small)) {
+  if (knob(kKnobTriTile) == 2 || (knob(kKnobTriTile) == 1 && (small || (sizeof(T) == 8 && upper)))) {
     bool handled = false;
     const int st = upper ? tt::tri_tile_run<T, true, true, TRI_UPPER, false, true>(l, a, lda, n, args.xc, incx, alpha, beta,
                                                                                   args.y, incy, &handled)
