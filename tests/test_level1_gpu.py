@@ -304,3 +304,35 @@ def test_level1_n_2_28(b2, ctx):
     assert_close(y3[tidx].cpu().numpy(), dtype(-0.75) * ox, ax, dtype, "swap + scal")  # 0.75 x the rot bound + one rounding
     b2.copy(ctx, n, dx, 1, x3, 1)
     assert torch.equal(x3, dx)
+
+
+def test_prepare_replays_the_recorded_calls(b2, ctx):
+    """binding.prepare marshals the calls of a thunk once; every replay must launch exactly those
+    calls again (same pointers, same scalars): axpy twice and a dot, checked against the oracle
+    after the recording run and after two replays."""
+    n = 70001
+    x = synth.vector_np(21, 1, n, np.float32)
+    y = synth.vector_np(21, 2, n, np.float32)
+    gx, gy = Guarded(x), Guarded(y)
+    res = torch.zeros(1, dtype=torch.float32, device="cuda")
+
+    def thunk():
+        b2.axpy(ctx, n, 0.5, gx.t, 1, gy.t, 1)
+        b2.axpy(ctx, n, -0.25, gx.t, 1, gy.t, 1)
+        b2.dot(ctx, n, gx.t, 1, gy.t, 1, res)
+
+    run = b2.prepare(thunk)  # runs the thunk once
+    oy = y.copy()
+    yabs = np.zeros(n)
+    launches = b2.launch_count()
+    for rounds in range(3):
+        if rounds:
+            assert run() == 0
+        a1 = orc.axpy(n, np.float32(0.5), x, 1, oy, 1)
+        a2 = orc.axpy(n, np.float32(-0.25), x, 1, oy, 1)
+        yabs = yabs + a1 + a2  # the error bound grows with every update of y
+        assert_close(gy.host(), oy, yabs, np.float32, f"axpy after {rounds} replays")
+        want, absterms = orc.dot(n, x, 1, oy, 1)
+        assert_close(res.cpu().numpy()[0], want, absterms, np.float32, f"dot after {rounds} replays")
+    assert b2.launch_count() - launches == 6  # two replays of three calls
+    gx.check_guards(), gy.check_guards()
