@@ -361,10 +361,15 @@ __global__ void __launch_bounds__(kThreads) l1_reduce_unit(const T* __restrict__
       const int64_t v0 = chunk * (int64_t)(kThreads * NV) + threadIdx.x;
       P px[NV];
       T m = T(-1);
+      if (v0 + (int64_t)(NV - 1) * kThreads < nvec) {  // every pack of the thread exists: plain loads
 #pragma unroll
-      for (int k = 0; k < NV; ++k) {
-        const int64_t v = v0 + (int64_t)k * kThreads;
-        px[k] = ld_nc_if<T, V>(xv + v * V, v < nvec);
+        for (int k = 0; k < NV; ++k) px[k] = ld_nc<T, V>(xv + (v0 + (int64_t)k * kThreads) * V);
+      } else {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+          const int64_t v = v0 + (int64_t)k * kThreads;
+          px[k] = ld_nc_if<T, V>(xv + v * V, v < nvec);
+        }
       }
 #pragma unroll
       for (int k = 0; k < NV; ++k) {
