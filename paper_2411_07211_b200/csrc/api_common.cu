@@ -12,10 +12,10 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobUsePdl          */ 1,
     /* kKnobTrsvDebugSkip   */ -1,
     /* kKnobTriWide         */ 0,
-    /* kKnobTrsvPrefetchBytes */ 48 << 20,
+    /* kKnobTrsvPrefetchBytes */ 12 << 20,
     /* kKnobTrsvFront       */ 2,
     /* kKnobTrsvCluster     */ 0,
-    /* kKnobTrsvPmFrom      */ 16,
+    /* kKnobTrsvPmFrom      */ -1,
     /* kKnobTriTile         */ 1,
     /* kKnobTriTileUnit     */ 0,
     /* kKnobNarrowBlock     */ 1,

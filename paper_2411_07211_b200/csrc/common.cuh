@@ -342,7 +342,7 @@ enum Knob {
   kKnobTrsvPrefetchBytes = 8,  // total L2 bytes trsv blocks may prefetch ahead of the front
   kKnobTrsvFront = 9,          // 0: block-row trsv kernel only; 1: sub-block kernel for row-type views; 2: for all views
   kKnobTrsvCluster = 10,       // sub-block trsv in clusters of 8 block rows: 0 never, 1 float only, 2 always
-  kKnobTrsvPmFrom = 11,        // first block row whose last tile is premultiplied by the inverse diagonal block
+  kKnobTrsvPmFrom = 11,        // first block row whose last tile is premultiplied by the inverse diagonal block (-1: by precision)
   kKnobTriTile = 12,           // tile kernel with the shared-memory ring: 0 never, 1 symv and the trmv cases it wins, 2 symv and every trmv
   kKnobTriTileUnit = 13,       // tiles per unit of that kernel: 0 = by size, else 1, 2 or 4
   kKnobNarrowBlock = 14,       // gemv on unpadded narrow matrices: 1 = block-wide kernels, 0 = warp-wide / general ones
