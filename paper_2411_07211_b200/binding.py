@@ -30,6 +30,7 @@ KNOB_GER_ROWS, KNOB_USE_PDL, KNOB_TRSV_DEBUG_SKIP, KNOB_TRI_WIDE = 4, 5, 6, 7
 KNOB_TRSV_PREFETCH_BYTES = 8
 KNOB_TRSV_FRONT, KNOB_TRSV_CLUSTER = 9, 10
 KNOB_TRSV_PM_FROM, KNOB_TRI_TILE, KNOB_TRI_TILE_UNIT, KNOB_NARROW_BLOCK = 11, 12, 13, 14
+KNOB_TRI_BULK = 15
 
 # B2BLAS_LIB selects another build of the same library (the bounds-checking one, libb2blas_dbg.so)
 LIB_PATH = os.environ.get("B2BLAS_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libb2blas.so")

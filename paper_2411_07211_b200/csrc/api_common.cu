@@ -19,6 +19,7 @@ static int64_t g_knobs[kKnobCount] = {
     /* kKnobTriTile         */ 1,
     /* kKnobTriTileUnit     */ 0,
     /* kKnobNarrowBlock     */ 1,
+    /* kKnobTriBulk         */ 0,
 };
 
 unsigned long long g_launch_count = 0;

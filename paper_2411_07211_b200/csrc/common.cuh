@@ -346,6 +346,7 @@ enum Knob {
   kKnobTriTile = 12,           // tile kernel with the shared-memory ring: 0 never, 1 symv and the trmv cases it wins, 2 symv and every trmv
   kKnobTriTileUnit = 13,       // tiles per unit of that kernel: 0 = by size, else 1, 2 or 4
   kKnobNarrowBlock = 14,       // gemv on unpadded narrow matrices: 1 = block-wide kernels, 0 = warp-wide / general ones
+  kKnobTriBulk = 15,           // tile kernel with the shared-memory ring: 1 = a tile arrives as one tiled TMA copy (measured equal to the 16-byte copies; off by default)
   kKnobCount = 16
 };
 int64_t knob(int id);

@@ -19,6 +19,8 @@
 // read it).
 #pragma once
 
+#include <cuda.h>  // CUtensorMap (types only: the encoder is fetched from the driver at run time)
+
 #include "level2.cuh"
 
 namespace b2 {
@@ -26,7 +28,10 @@ namespace tt {
 
 // (measured: wider, flatter tiles -- 64 x 256 or 32 x 512 floats -- are slower here, they waste
 // more of the tiles that the diagonal cuts and make the units coarser)
-constexpr int kRing = 3;       // tiles (64 KB each) in the shared-memory ring
+#ifndef B2_TT_RING
+#define B2_TT_RING 3
+#endif
+constexpr int kRing = B2_TT_RING;  // tiles (64 KB each at 128 rows) in the shared-memory ring
 #ifndef B2_TT_NR
 #define B2_TT_NR 8
 #endif
@@ -72,6 +77,7 @@ struct TileArgs {
   T alpha, beta;
   T* y;
   int64_t incy;
+  int* status;  // device status word (may be null): a bounded wait that ran out reports here
   int prefix[CAP + 1];  // units before block row (column tile) i; the last entry is their total
 };
 
@@ -112,6 +118,39 @@ __device__ __forceinline__ void cp_async_elem(void* dst, const void* src, bool v
                "n"(N), "r"(valid ? N : 0)
                : "memory");
 }
+// Bulk asynchronous copies (one instruction per contiguous run, no per-thread load path) and the
+// shared-memory barrier that counts their bytes.  Source and destination 16-byte aligned, size a
+// multiple of 16; this GPU's own memory, no multicast.
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect(unsigned long long* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+  unsigned done;
+  asm volatile(
+      "{\n\t.reg .pred q;\n\tmbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(done)
+      : "r"((unsigned)__cvta_generic_to_shared(bar)), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, unsigned bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   (unsigned)__cvta_generic_to_shared(dst)),
+               "l"(src), "r"(bytes), "r"((unsigned)__cvta_generic_to_shared(bar))
+               : "memory");
+}
+// One tiled TMA copy: the box of the tensor map at element coordinates (x, y) -> shared memory.
+// x * element size must be a multiple of 16 bytes; what lies outside the tensor arrives as zeros.
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+                   (unsigned)__cvta_generic_to_shared(dst)),
+               "l"(map), "r"(x), "r"(y), "r"((unsigned)__cvta_generic_to_shared(bar))
+               : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
@@ -125,20 +164,36 @@ __device__ __forceinline__ void cp_async_wait() {
 // next kRing - 1 tiles (also those of the block's next units) are in flight while a tile is
 // multiplied.  Edge tiles use the same copies with a byte count that zero-fills what lies outside
 // the matrix.  The x values of a unit travel the same way.
-template <typename T, int CAP, bool ROW, bool COL, int TRI, bool UNIT, bool SYM>
-__global__ void __launch_bounds__(kThreads, kBlocksPerSm) tri_tile_kernel(const TileArgs<T, CAP> p) {
+// BULK: a tile arrives as ONE tiled TMA copy (tensor map over the n x n matrix, box = one tile;
+// what lies outside the matrix arrives as zeros), issued by one thread and counted by a
+// shared-memory barrier per ring slot, and lies row-major in its slot; one block-wide barrier per
+// tile keeps the refill of a slot behind its last reader.  Every wait on a barrier is bounded.
+// (kTR separate row-sized bulk copies per tile measured three times SLOWER than the 16-byte
+// per-thread copies: the fixed cost of a bulk copy is paid per 512 bytes.)
+template <typename T, int CAP, bool ROW, bool COL, int TRI, bool UNIT, bool SYM, bool BULK = false>
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm) tri_tile_kernel(const TileArgs<T, CAP> p, const __grid_constant__ CUtensorMap tmap) {
   constexpr int V = VecLen<T>::value, TC = 16 * kNP * V, NR = kNR, HR = NR / 2, NP = kNP, TP = NR * NP;
   constexpr bool WALK_ROWS = ROW;  // column-sum-only kinds walk down a block column
   constexpr int XCU = WALK_ROWS ? kUnitMax * TC : TC;  // most column values a unit needs
   using P = Pack<T, V>;
   grid_dep_wait();
   grid_dep_launch();
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   uint4* ring = reinterpret_cast<uint4*>(smem_raw);             // [kRing][TP][kThreads] packs
   T* xr_q = reinterpret_cast<T*>(ring + kRing * TP * kThreads);  // [slots] row values of the units in flight
   constexpr int XRQ = COL ? kSlotElems<T, WALK_ROWS, true>() : 0, XCQ = ROW ? kSlotElems<T, WALK_ROWS, false>() : 0;
   T* xc_q = xr_q + XRQ;  // [slots] column values
   T* cbuf = xc_q + XCQ;  // [kWarps][XCU] column sums of the warps
+  __shared__ unsigned long long full_bar[kRing];
+  if (BULK) {
+    if (threadIdx.x == 0) {
+      for (int s = 0; s < kRing; ++s) mbar_init(&full_bar[s], 1u);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+  }
+  unsigned bar_phase = 0;  // bit s: parity of the next completion of slot s
+  bool dead = false;       // a bounded wait ran out: drain without touching the tiles
 
   const int ct = (int)threadIdx.x, warp = ct >> 5, lane = ct & 31;
   const int rg = ct >> 4, cg = ct & 15;
@@ -204,7 +259,12 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) tri_tile_kernel(const 
       }
       uint4* dst = ring + (size_t)pstage * TP * kThreads + ct;
       const T* src = p.a + r0 * p.lda + c0 + thread_off;
-      if (r0 + kTR <= p.n && c0 + TC <= p.n) {
+      if (BULK) {
+        if (ct == 0) {
+          mbar_arrive_expect(&full_bar[pstage], (unsigned)(kTR * TC * sizeof(T)));
+          tma_load_2d(ring + (size_t)pstage * TP * kThreads, &tmap, (int)c0, (int)r0, &full_bar[pstage]);
+        }
+      } else if (r0 + kTR <= p.n && c0 + TC <= p.n) {
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -245,13 +305,29 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) tri_tile_kernel(const 
   for (int s = 0; s < kRing - 1; ++s) produce();
 #pragma unroll 1
   while (cons.valid) {
+    if (BULK) __syncthreads();  // every thread has left the slot that this trip's copies refill
     produce();
     cp_async_wait<kRing - 1>();  // this thread's copies of the oldest tile in flight have landed
+    if (BULK && !dead) {  // ... and so has the tile itself (bounded: a wait that runs out is reported, the block drains)
+      const unsigned parity = (bar_phase >> cstage) & 1u;
+      bool ok = false;
+      for (int spin = 0; spin < (1 << 22) && !ok; ++spin) ok = mbar_try_wait(&full_bar[cstage], parity);
+      bar_phase ^= 1u << cstage;
+      if (!ok) {
+        dead = true;
+        if (p.status) atomicExch(p.status, (int)B2_STATUS_TIMEOUT);
+      }
+    }
     const int I = WALK_ROWS ? cons.major : cons.t, J = WALK_ROWS ? cons.t : cons.major;
     const int I0 = WALK_ROWS ? I : cons.t0, J0 = WALK_ROWS ? cons.t0 : J;
     if (cons.t == cons.t0) __syncthreads();  // the unit's x values came from other threads' copies
     const int64_t r0 = (int64_t)I * kTR, c0 = (int64_t)J * TC;
-    const uint4* src = ring + (size_t)cstage * TP * kThreads + ct;
+    // the thread's packs of the tile: its own copies (one slot entry per pack and thread), or, in a
+    // tile that came as whole rows, row (h, a) of its row group and the packs cg, cg + 16 of that row
+    const uint4* src = ring + (size_t)cstage * TP * kThreads + (BULK ? (rg * HR) * (TC / V) + cg : ct);
+    auto pack_at = [&](int h, int a, int hb) -> int {
+      return BULK ? (h * (kTR / 2) + a) * (TC / V) + hb * 16 : ((h * HR + a) * NP + hb) * kThreads;
+    };
     cstage = cstage + 1 == kRing ? 0 : cstage + 1;
     T xc[NP][V];
     if (ROW) {
@@ -273,7 +349,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) tri_tile_kernel(const 
       for (int a = 0; a < HR; ++a)
 #pragma unroll
         for (int hb = 0; hb < NP; ++hb) {
-          const uint4 raw = src[((h * HR + a) * NP + hb) * kThreads];
+          const uint4 raw = dead ? make_uint4(0u, 0u, 0u, 0u) : src[pack_at(h, a, hb)];
           const P pk = *reinterpret_cast<const P*>(&raw);
 #pragma unroll
           for (int e = 0; e < V; ++e) m[a][hb][e] = pk.v[e];
@@ -354,6 +430,11 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) tri_tile_kernel(const 
     advance(cons);
   }
   cp_async_wait<0>();
+  if (BULK && dead) {  // copies may still be on their way into this block's shared memory: give them time to land
+    for (int s = 0; s < kRing; ++s)
+      for (int spin = 0; spin < (1 << 16) && !mbar_try_wait(&full_bar[s], (bar_phase >> s) & 1u); ++spin) {
+      }
+  }
 }
 
 // y_i = alpha * (row partials of i + column partials of i) + beta * y_i, the partials added in a
@@ -424,6 +505,34 @@ constexpr size_t tile_smem_bytes() {
                               (COL ? kWarps * (WALK_ROWS ? kUnitMax * TC : TC) : 0));
 }
 
+// Tensor map of the n x n row-major matrix with boxes of one tile (kTR rows x tc columns).  The
+// encoder lives in the driver; it is looked up once.  false: no encoder, or the matrix does not
+// meet the map's rules (the caller then uses the 16-byte copies).
+template <typename T>
+static bool encode_tile_map(CUtensorMap* map, const T* a, int64_t lda, int64_t n, int tc) {
+  using Encode = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static Encode encode = [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) {
+      (void)cudaGetLastError();
+      fn = nullptr;
+    }
+    return reinterpret_cast<Encode>(fn);
+  }();
+  if (encode == nullptr) return false;
+  if ((lda * sizeof(T)) % 16 != 0 || !aligned_to(a, 16)) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)n};
+  const cuuint64_t strides[1] = {(cuuint64_t)lda * sizeof(T)};
+  const cuuint32_t box[2] = {(cuuint32_t)tc, (cuuint32_t)kTR};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapDataType dt = sizeof(T) == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT64;
+  return encode(map, dt, 2, const_cast<T*>(a), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Launches both kernels.  *handled is false (nothing launched) when the matrix is not 16-byte
 // aligned, too large for the unit table, or the partials do not fit the workspace: the caller
 // then uses the general tile kernel.
@@ -469,8 +578,17 @@ static int tri_tile_run_cap(const Launch& l, const T* a, int64_t lda, int64_t n,
   args.beta = beta;
   args.y = y;
   args.incy = incy;
+  args.status = l.device_status;
   constexpr size_t smem = tile_smem_bytes<T, ROW, COL>();
-  auto kern = tri_tile_kernel<T, CAP, ROW, COL, TRI, UNIT, SYM>;
+  // whole rows by bulk copies when every tile is full (and the rows' starts and lengths are then
+  // multiples of 16 bytes, which those copies need)
+  CUtensorMap tmap = {};
+  bool bulk = knob(kKnobTriBulk) != 0 && n <= 0x7fffffff;
+#ifdef B2_DEBUG_BOUNDS
+  bulk = false;  // (a TMA copy cannot be tested address by address: the checking build keeps the 16-byte copies)
+#endif
+  if (bulk) bulk = encode_tile_map<T>(&tmap, a, lda, n, TC);
+  auto kern = bulk ? tri_tile_kernel<T, CAP, ROW, COL, TRI, UNIT, SYM, true> : tri_tile_kernel<T, CAP, ROW, COL, TRI, UNIT, SYM, false>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     (void)cudaGetLastError();
     return B2_STATUS_OK;
@@ -478,7 +596,7 @@ static int tri_tile_run_cap(const Launch& l, const T* a, int64_t lda, int64_t n,
   *handled = true;
   const int nunits = args.prefix[nmajor];
   const int grid = nunits < sm_count() * kBlocksPerSm ? nunits : sm_count() * kBlocksPerSm;
-  launch_chained(kern, dim3(grid), dim3(kThreads), smem, l.stream, args);
+  launch_chained(kern, dim3(grid), dim3(kThreads), smem, l.stream, args, tmap);
   if (int st = check_launch()) return st;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)((n + 31) / 32));

@@ -382,7 +382,7 @@ def test_symv_trmv_every_unit_length(b2, ctx, dtype, unit):
     b2.set_tuning(b2.KNOB_TRI_TILE_UNIT, unit)
     b2.set_tuning(b2.KNOB_TRI_TILE, 2)  # every trmv through the tile kernel too
     try:
-        for n in (700, 2443):
+        for n in (700, 2443, 1280, 2560):  # (the last two: every tile full)
             a = synth.matrix_np(17, 3, n, n, n, dtype, tri_n=n).ravel()
             x, y = synth.vector_np(17, 4, n, dtype), synth.vector_np(17, 5, n, dtype)
             ga = Guarded(a)
@@ -401,6 +401,40 @@ def test_symv_trmv_every_unit_length(b2, ctx, dtype, unit):
     finally:
         b2.set_tuning(b2.KNOB_TRI_TILE_UNIT, old[0])
         b2.set_tuning(b2.KNOB_TRI_TILE, old[1])
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_tile_kernel_tma_delivery(b2, ctx, dtype):
+    """The ring kernel with its tiles delivered by one tiled TMA copy each (tensor map over the
+    matrix, zero fill outside it, a shared-memory barrier per ring slot with bounded waits): symv
+    and every trmv on sizes with ragged edges, with only full tiles, and with more units than SMs;
+    the device status must stay clean (a barrier wait that ran out would set it)."""
+    old = b2.get_tuning(b2.KNOB_TRI_TILE), b2.get_tuning(b2.KNOB_TRI_BULK)
+    b2.set_tuning(b2.KNOB_TRI_TILE, 2)
+    b2.set_tuning(b2.KNOB_TRI_BULK, 1)
+    try:
+        for n, pad in ((130, 0), (700, 4), (1280, 0), (2443, 0), (2560, 8)):
+            lda = n + pad
+            a = synth.matrix_np(19, 3, n, lda, lda, dtype, tri_n=n).ravel()
+            x, y = synth.vector_np(19, 4, n, dtype), synth.vector_np(19, 5, n, dtype)
+            ga = Guarded(a)
+            for uplo in UPLOS:
+                gx, gy = Guarded(x), Guarded(y)
+                b2.symv(ctx, orc.ROW_MAJOR, uplo, n, 1.25, ga.t, lda, gx.t, 1, 0.5, gy.t, 1)
+                oy = y.copy()
+                absterms = orc.symv(orc.ROW_MAJOR, uplo, n, dtype(1.25), a, lda, x, 1, dtype(0.5), oy, 1)
+                assert_close(gy.host(), oy, absterms, dtype, f"symv n={n} uplo={uplo}")
+                for trans, diag in itertools.product(TRANSES, DIAGS):
+                    gx = Guarded(x)
+                    b2.trmv(ctx, orc.ROW_MAJOR, uplo, trans, diag, n, ga.t, lda, gx.t, 1)
+                    ox = x.copy()
+                    absterms = orc.trmv(orc.ROW_MAJOR, uplo, trans, diag, n, a, lda, ox, 1)
+                    assert_close(gx.host(), ox, absterms, dtype, f"trmv n={n} {uplo} {trans} {diag}")
+            assert ctx.device_status() == 0
+            ga.check_guards()
+    finally:
+        b2.set_tuning(b2.KNOB_TRI_TILE, old[0])
+        b2.set_tuning(b2.KNOB_TRI_BULK, old[1])
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
