@@ -46,7 +46,7 @@ enum {
   B2_STATUS_LAUNCH_FAILED = 1,       /* a CUDA launch or memset was rejected (error consumed)   */
   B2_STATUS_WORKSPACE_TOO_SMALL = 2, /* ctx->workspace_bytes below what this call needs          */
   B2_STATUS_NOT_IMPLEMENTED = 3,
-  B2_STATUS_TIMEOUT = 4,             /* only ever written to *ctx->device_status (trsv waits)    */
+  B2_STATUS_TIMEOUT = 4,             /* only ever written to *ctx->device_status (bounded waits) */
   B2_STATUS_BAD_CONTEXT = 5,         /* ctx NULL, workspace NULL / misaligned                    */
   B2_STATUS_TOO_LARGE = 6            /* problem size above the fixed limit of a *_noalloc call   */
 };
@@ -65,7 +65,9 @@ enum {
  *                   Never written otherwise; the caller zeroes it.  A timed-out call leaves
  *                   the control block dirty: call b2_workspace_reset before the workspace is
  *                   used again.  A trsv call that finds the control block dirty solves
- *                   nothing and writes B2_STATUS_TIMEOUT again.
+ *                   nothing and writes B2_STATUS_TIMEOUT again.  (symv / trmv write the same
+ *                   value only with the optional TMA tile delivery switched on, if a wait
+ *                   for a copy into shared memory ran out; they keep no state.)
  *   wait_limit      polling iterations before a trsv wait gives up; 0 = library default.
  */
 typedef struct b2_ctx {
